@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark: one step = the 53 convolutions of ResNet-50 v1 at batch 64, the
+depthwise case and the classifier-head Gemm, each launched once through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is TFLOP/s over the whole step with inputs resident
+in HBM; `e2e` repeats the measurement with host (pinned) inputs copied in and the
+outputs copied back inside the timed region.  `--impl reference` times the fp64
+CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2008_08272_b200 import workloads as wl  # noqa: E402
+
+METRIC = "Conv/Gemm TFLOP/s (fp32 I/O, TF32 MMA)"
+WORKLOAD = "resnet50_v1_53conv_sweep_b64+depthwise_256x28x28+gemm_head_64x1000x2048"
+TF32_OVER_BF16 = 1125.0 / 2250.0     # nominal dense ratio, applied to the measured bf16 peak
+SAMPLE_IMAGES = 4
+SAMPLE_TEXT = ("first 4 images of each of the 54 convolutions plus the full head Gemm "
+               "(1/16 of a step's convolution work)")
+FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max clock
+
+
+def step_ops(batch: int = 64):
+    """The ops of one step, in launch order."""
+    convs = wl.resnet50_v1_convs(batch) + [wl.config5_depthwise(batch)]
+    gemm = wl.GemmCase("r50_head_gemm", (batch, 2048), (1000, 2048), (1000,), transB=True,
+                       seed=wl.SEED_BASE + 1000 * 5 + 54)
+    return convs, gemm
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"],
+                    bf16_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs (read-only query)."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_reference(args):
+    """The fp64 CPU oracle, as it stands, on a bounded sample of the step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    convs, gemm = step_ops()
+    sample = SAMPLE_TEXT
+    prepared = []
+    for c in convs:
+        X, W, B = wl.conv_inputs(wl.with_batch(c, SAMPLE_IMAGES))
+        prepared.append((c, X, W, B))
+    A, Bm, C = wl.gemm_inputs(gemm)
+    flops = sum(wl.with_batch(c, SAMPLE_IMAGES).flops for c in convs) + gemm.flops
+
+    def one():
+        for c, X, W, B in prepared:
+            oracle.conv2d(X, W, B, pads=c.pads, strides=c.strides, dilations=c.dilations, group=c.group,
+                          relu=c.relu, want_s=False)
+        oracle.gemm(A, Bm, C, transB=True, want_s=False)
+
+    for _ in range(min(args.warmup, 1)):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = flops / dt / 1e12
+    cores = oracle.threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch": 64, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2008_08272_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load(build_if_missing=False)
+
+    convs, gemm = step_ops()
+    # ---- inputs: seeded host arrays (pinned, reused by the e2e leg) and resident device copies
+    host, devt, descs = [], [], []
+    for c in convs:
+        X, W, B = wl.conv_inputs(c)
+        hx, hw, hb = (torch.from_numpy(t).pin_memory() for t in (X, W, B))
+        host.append((hx, hw, hb))
+        d = binding.Conv2dDesc(c.x_shape, c.w_shape, pads=c.pads, strides=c.strides, dilations=c.dilations,
+                               group=c.group, has_bias=True, fuse_relu=c.relu)
+        ws = torch.empty(max(d.workspace_bytes, 16), dtype=torch.uint8, device=dev)
+        y = torch.empty(d.y_shape, dtype=torch.float32, device=dev)
+        devt.append([hx.to(dev), hw.to(dev), hb.to(dev), y, ws])
+        descs.append(d)
+    A, Bm, C = wl.gemm_inputs(gemm)
+    g_host = tuple(torch.from_numpy(t).pin_memory() for t in (A, Bm, C))
+    g_dev = [t.to(dev) for t in g_host]
+    gm, gn, gk = gemm.mnk
+    g_y = torch.empty((gm, gn), dtype=torch.float32, device=dev)
+    g_ws = torch.empty(max(binding.gemm_workspace_bytes(False, True, gm, gn, gk), 16), dtype=torch.uint8, device=dev)
+    y_host = torch.empty(max(int(np.prod(d.y_shape)) for d in descs), dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+
+    flops_per_step = sum(c.flops for c in convs) + gemm.flops
+    bytes_per_op = [c.algorithmic_bytes for c in convs] + [4 * (gm * gk + gn * gk + gn + gm * gn)]
+    flops_per_op = [c.flops for c in convs] + [gemm.flops]
+    families = [d.kernel_family for d in descs] + ["gemm"]
+    n_ops = len(flops_per_op)
+
+    def launch_all(events=None):
+        for i, d in enumerate(descs):
+            x, w, b, y, ws = devt[i]
+            d.run(x, w, b, Y=y, workspace=ws)
+            if events is not None:
+                events[i + 1].record()
+        binding.onnx_gemm(g_dev[0], g_dev[1], g_dev[2], transB=True, Y=g_y, workspace=g_ws)
+        if events is not None:
+            events[n_ops].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        launch_all()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ops + 1)] for _ in range(args.steps)]
+    launches0 = binding.launch_count()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for s in range(args.steps):
+        ev[s][0].record()
+        launch_all(ev[s])
+    t_end.record()
+    barrier()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t_start.elapsed_time(t_end)
+    assert binding.last_device_status() == 0, "a device-side wait timed out"
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+    # per-op durations (same timed region), grouped by kernel family
+    per_op_ms = [statistics.fmean(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps))
+                 for i in range(n_ops)]
+    fam_time, fam_flops, fam_bytes, fam_count = {}, {}, {}, {}
+    for i, f in enumerate(families):
+        fam_time[f] = fam_time.get(f, 0.0) + per_op_ms[i]
+        fam_flops[f] = fam_flops.get(f, 0) + flops_per_op[i]
+        fam_bytes[f] = fam_bytes.get(f, 0) + bytes_per_op[i]
+        fam_count[f] = fam_count.get(f, 0) + 1
+    top = max(fam_time, key=fam_time.get)
+    peaks = measured_peaks()
+    tensor_peak = peaks["bf16_sustained"] * TF32_OVER_BF16
+    ach_tflops = fam_flops[top] / (fam_time[top] * 1e-3) / 1e12
+    ach_gbs = fam_bytes[top] / (fam_time[top] * 1e-3) / 1e9
+    if top.startswith("mma"):
+        # a dense contraction fed from HBM: report the roof that binds this family's aggregate
+        t_tensor = fam_flops[top] / (tensor_peak * 1e12)
+        t_hbm = fam_bytes[top] / (peaks["hbm_gbs"] * 1e9)
+        if t_tensor >= t_hbm:
+            roof = {"bound": "tensor", "achieved": ach_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
+                    "frac": ach_tflops / tensor_peak}
+        else:
+            roof = {"bound": "hbm", "achieved": ach_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach_gbs / peaks["hbm_gbs"]}
+        roof["peak_source"] = (f"{peaks['source']} bf16 sustained x nominal tf32/bf16 ratio 0.5"
+                               if roof["bound"] == "tensor" else f"{peaks['source']} HBM copy")
+    elif top == "simt_depthwise":
+        roof = {"bound": "hbm", "achieved": ach_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach_gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} HBM copy"}
+    else:
+        roof = {"bound": "alu", "achieved": ach_tflops, "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s",
+                "frac": ach_tflops / FP32_FMA_PEAK_TFLOPS,
+                "peak_source": "derived: 148 SMs x 128 fp32 FMA/clk x 2 x 1.965 GHz"}
+    roof.update({"kernel": top, "launches_per_step": fam_count[top], "ms_per_step": fam_time[top],
+                 "traffic": None})
+    families_out = {f: {"ops": fam_count[f], "ms": round(fam_time[f], 4),
+                        "tflops": round(fam_flops[f] / (fam_time[f] * 1e-3) / 1e12, 3),
+                        "gbs": round(fam_bytes[f] / (fam_time[f] * 1e-3) / 1e9, 1)} for f in fam_time}
+
+    # ---- end to end: pinned host inputs in, results out, every step
+    e2e_steps = max(1, min(args.steps, 2))
+    h2d = sum(t.numel() * 4 for trip in host for t in trip) + sum(t.numel() * 4 for t in g_host)
+    d2h = sum(int(np.prod(d.y_shape)) * 4 for d in descs) + gm * gn * 4
+
+    def e2e_step():
+        for i, d in enumerate(descs):
+            hx, hw, hb = host[i]
+            x, w, b, y, ws = devt[i]
+            x.copy_(hx, non_blocking=True)
+            w.copy_(hw, non_blocking=True)
+            b.copy_(hb, non_blocking=True)
+            d.run(x, w, b, Y=y, workspace=ws)
+            y_host[: y.numel()].copy_(y.view(-1), non_blocking=True)
+        for dt_, ht_ in zip(g_dev, g_host):
+            dt_.copy_(ht_, non_blocking=True)
+        binding.onnx_gemm(g_dev[0], g_dev[1], g_dev[2], transB=True, Y=g_y, workspace=g_ws)
+        y_host[: g_y.numel()].copy_(g_y.view(-1), non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * flops_per_step / (e2e_ms * 1e-3) / 1e12
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, single GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        sample_flops, t_cpu = 0, 0.0
+        for i, c in enumerate(convs):
+            hx, hw, hb = host[i]
+            X1 = hx[:SAMPLE_IMAGES].numpy()
+            t0 = time.perf_counter()
+            oracle.conv2d(X1, hw.numpy(), hb.numpy(), pads=c.pads, strides=c.strides, dilations=c.dilations,
+                          group=c.group, relu=c.relu, want_s=False)
+            t_cpu += time.perf_counter() - t0
+            sample_flops += wl.with_batch(c, SAMPLE_IMAGES).flops
+        t0 = time.perf_counter()
+        oracle.gemm(A, Bm, C, transB=True, want_s=False)
+        t_cpu += time.perf_counter() - t0
+        sample_flops += gemm.flops
+        cpu = {"value": sample_flops / t_cpu / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(),
+               "kind": "oracle", "seconds": round(t_cpu, 3),
+               "sample": SAMPLE_TEXT}
+
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return 0
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "tf32" if any(f.startswith("mma") for f in families) else "f32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": 64, "ops_per_step": n_ops,
+                   "gflop_per_step": round(flops_per_step / 1e9, 3),
+                   "l2": "inputs larger than L2: every op has its own X/W/Y buffers, ~8 GB touched per step",
+                   "parallelism": f"replicas x{world} (batch split, no collective)"},
+        "pct_of_nominal_tf32_peak_1125": round(100 * value / world / 1125.0, 2),
+        "roofline": roof, "kernel_families": families_out,
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,194 @@
+/*
+ * onnx_b200.h - C ABI of the ONNX Conv / Gemm library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the two operators at the centre of the inference code an
+ * ONNX compiler emits for MNIST- and ResNet-50-class models (the paper's Sec. 4.1
+ * names convolution and Gemm as supported operators; Sec. 4.2 runs both models):
+ * ONNX Conv (2-D, NCHW) and ONNX Gemm, each with a fused bias and an optional
+ * fused Relu (the producer/consumer fusion idea of Sec. 3.4.3).  Operator
+ * semantics follow the ONNX standard the paper builds on (Sec. 2.1); shapes are
+ * inferred from input shapes and attributes as in the shape-inference pass of
+ * Sec. 3.4.2, restricted to static shapes.
+ *
+ * General conventions
+ *   - All tensors are dense, row-major, 32-bit float.  Conv tensors are NCHW.
+ *   - Pointers named X, W, B, A, C, Y and `workspace` are DEVICE pointers owned
+ *     by the caller.  Attribute structs, dims arrays and out-parameters are HOST
+ *     memory.  `cuda_stream` is a cudaStream_t passed as void* (NULL = the
+ *     default stream).
+ *   - Run calls enqueue work on the given stream and return without
+ *     synchronising.  They never allocate or free device memory.
+ *   - Inputs are read-only; Y must not overlap any input or the workspace.
+ *   - Every device pointer must be 16-byte aligned.
+ *   - No C++ exception crosses this boundary; every failure is a status code and
+ *     leaves Y untouched (errors are detected before anything is launched).
+ *   - Tensors with more than 2^31-1 elements are rejected (ONNXB_ERR_UNSUPPORTED).
+ *   - Arithmetic: fp32 inputs and outputs.  Kernels of the tensor-core family
+ *     multiply in TF32 (10-bit mantissa operands) and accumulate in fp32; kernels
+ *     of the SIMT family use fp32 FMA.  Either way
+ *         |Y - exact| <= 1e-3 * sum|x*w| + 1e-5       per output element
+ *     for finite inputs of moderate magnitude.
+ */
+#ifndef ONNX_B200_H_
+#define ONNX_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ONNXB_OK = 0,
+    ONNXB_ERR_NULL = 1,            /* a required pointer is NULL (or B given/omitted against has_bias) */
+    ONNXB_ERR_ATTR = 2,            /* an attribute value ONNX does not admit */
+    ONNXB_ERR_SHAPE = 3,           /* shapes inconsistent with each other or with the attributes */
+    ONNXB_ERR_UNSUPPORTED = 4,     /* valid ONNX, outside this library's range (size, alignment, negative pads) */
+    ONNXB_ERR_WORKSPACE = 5,       /* workspace missing or smaller than the descriptor asks for */
+    ONNXB_ERR_CUDA = 6,            /* a CUDA runtime/driver call failed (launch configuration, no device) */
+    ONNXB_ERR_DEVICE_TIMEOUT = 7   /* a bounded device-side wait ran out (see onnxb_last_device_status) */
+} onnxb_status;
+
+typedef enum {
+    ONNXB_NOTSET = 0,              /* use `pads` */
+    ONNXB_SAME_UPPER = 1,          /* out = ceil(in/stride); odd padding unit at the end */
+    ONNXB_SAME_LOWER = 2,          /* out = ceil(in/stride); odd padding unit at the beginning */
+    ONNXB_VALID = 3                /* no padding */
+} onnxb_auto_pad;
+
+/* Kernel family a descriptor resolved to (reported by onnx_conv2d_desc_query_kernel). */
+typedef enum {
+    ONNXB_KERNEL_SIMT_DIRECT = 0,  /* fp32 FMA direct convolution (thin contractions, any attributes) */
+    ONNXB_KERNEL_SIMT_DEPTHWISE = 1, /* fp32 FMA, one input channel per output channel, smem row tiles */
+    ONNXB_KERNEL_MMA_GEMM = 2,     /* 1x1 stride-1: batched tcgen05 TF32 GEMM straight from NCHW via TMA */
+    ONNXB_KERNEL_MMA_IMPLICIT = 3  /* general implicit GEMM: TMA staging + in-smem im2col + tcgen05 TF32 */
+} onnxb_kernel_family;
+
+/*
+ * Attribute set of ONNX Conv, one field per ONNX attribute (the paper's onnx
+ * dialect mirrors ONNX attributes one for one, Sec. 3.2), plus the two fusion
+ * switches.  Zero-initialise the struct to get every ONNX default.
+ */
+typedef struct {
+    int64_t x_dims[4];        /* N, C, H, W */
+    int64_t w_dims[4];        /* M, C/group, kH, kW */
+    int64_t kernel_shape[2];  /* {0,0}: infer from w_dims; otherwise must equal w_dims[2..3] */
+    int64_t pads[4];          /* ONNX order: h_begin, w_begin, h_end, w_end; >= 0 */
+    int64_t strides[2];       /* along H, along W; {0,0} = default {1,1} */
+    int64_t dilations[2];     /* along H, along W; {0,0} = default {1,1} */
+    int64_t group;            /* 0 = default 1 */
+    int32_t auto_pad;         /* onnxb_auto_pad; anything but NOTSET excludes non-zero pads */
+    int32_t has_bias;         /* non-zero: B[M] is added */
+    int32_t fuse_relu;        /* non-zero: max(.,0) applied to the result */
+    int32_t reserved;         /* must be 0 */
+} onnxb_conv2d_attrs;
+
+typedef struct onnxb_conv2d_desc_s *onnxb_conv2d_desc_t;
+
+/*
+ * onnx_conv2d_desc - validate attributes, resolve auto_pad, infer the output
+ * shape (Sec. 3.4.2) and choose a kernel (host only, no CUDA call).
+ *
+ *   P = floor((H + h_begin + h_end - ((kH-1)*dh + 1)) / sh) + 1, likewise Q.
+ *   SAME_*: P = ceil(H/sh), total = max((P-1)*sh + (kH-1)*dh + 1 - H, 0),
+ *           UPPER: begin = total/2, end = total - begin; LOWER the other way.
+ *
+ * attrs (host, read) ; out (host, written on success; destroy with
+ * onnx_conv2d_desc_destroy).  Descriptors are immutable and may be shared by
+ * threads.  Errors: NULL arguments -> ERR_NULL; non-positive stride/dilation,
+ * unknown auto_pad, auto_pad with non-zero pads, kernel_shape != W dims,
+ * reserved != 0 -> ERR_ATTR; non-positive dims, C % group, M % group,
+ * w_dims[1] != C/group, kernel larger than the padded input -> ERR_SHAPE;
+ * negative pads or a tensor above 2^31-1 elements -> ERR_UNSUPPORTED.
+ */
+onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *attrs, onnxb_conv2d_desc_t *out);
+
+/*
+ * onnx_conv2d_desc_query - read back what the descriptor resolved.  Any of the
+ * out-pointers (host) may be NULL.  y_dims = {N, M, P, Q}; resolved_pads in ONNX
+ * order; workspace_bytes = device scratch onnx_conv2d_run needs (may be 0).
+ */
+onnxb_status onnx_conv2d_desc_query(onnxb_conv2d_desc_t desc, int64_t y_dims[4],
+                                    int64_t resolved_pads[4], size_t *workspace_bytes);
+
+/* Kernel family the descriptor will launch (the dispatch step: a contraction of
+ * C/group*kH*kW terms that is too thin for the tensor cores, or a depthwise
+ * convolution, goes to a SIMT kernel).  Returns -1 for a NULL descriptor. */
+int onnx_conv2d_desc_query_kernel(onnxb_conv2d_desc_t desc);
+
+/*
+ * onnx_conv2d_run - Y = relu?( conv(X, W) + B ), ONNX Conv (Sec. 4.1), i.e.
+ *
+ *   Y[n,m,p,q] = B[m] + sum_{c<C/g, r<kH, s<kW}
+ *       Xpad[n, (m div (M/g))*(C/g)+c, p*sh + r*dh - h_begin, q*sw + s*dw - w_begin] * W[m,c,r,s]
+ *
+ * with Xpad = X inside the image and 0 outside; the kernel is not flipped.
+ *
+ * X [N,C,H,W], W [M,C/g,kH,kW], B [M] (NULL exactly when has_bias == 0),
+ * Y [N,M,P,Q]: device, fp32, dense.  workspace: device scratch of at least the
+ * queried size (NULL allowed when that size is 0); its contents are undefined on
+ * return and two runs that share a workspace must not overlap in time.
+ * Errors: ERR_NULL, ERR_WORKSPACE, ERR_UNSUPPORTED (misaligned pointer),
+ * ERR_CUDA (launch failure).
+ */
+onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t desc, const float *X, const float *W,
+                             const float *B, float *Y, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream);
+
+void onnx_conv2d_desc_destroy(onnxb_conv2d_desc_t desc);
+
+/*
+ * onnx_gemm_workspace_bytes - device scratch onnx_gemm_run needs for this
+ * problem (0 when none).  Host only.
+ */
+size_t onnx_gemm_workspace_bytes(int transA, int transB, int64_t M, int64_t N, int64_t K);
+
+/*
+ * onnx_gemm_run - ONNX Gemm (Sec. 3.4.3: Gemm(m1,m2,m3) = Add(MatMul(m1,m2),m3)):
+ *
+ *   Y[i,j] = relu?( alpha * sum_k A'[i,k] * B'[k,j] + beta * Cb[i,j] )
+ *
+ * A' = transA ? A^T : A is M x K (A stored [M,K], or [K,M] when transA != 0);
+ * B' = transB ? B^T : B is K x N (B stored [K,N], or [N,K] when transB != 0);
+ * Cb is C broadcast one-directionally to [M,N].  C == NULL omits the term;
+ * otherwise c_rank in {0,1,2} and c_dims (host) hold its shape: (), (1), (N),
+ * (1,N), (M,1), (1,1) or (M,N); a 1-D C is per column.  Y [M,N].
+ * Errors: ERR_NULL; ERR_SHAPE (M,N,K < 1, C shape not broadcastable);
+ * ERR_UNSUPPORTED (size, alignment); ERR_WORKSPACE; ERR_CUDA.
+ */
+onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float beta,
+                           int64_t M, int64_t N, int64_t K,
+                           const float *A, const float *B,
+                           const float *C, int c_rank, const int64_t *c_dims,
+                           int fuse_relu, float *Y, void *workspace, size_t workspace_bytes,
+                           void *cuda_stream);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char *onnxb_status_string(onnxb_status status);
+
+/*
+ * onnxb_last_device_status - every device-side wait in the tensor-core kernels
+ * is bounded; a wait that runs out sets an error word in device memory and the
+ * kernel drains and returns.  This call synchronises `cuda_stream`, reads and
+ * clears that word and returns ONNXB_ERR_DEVICE_TIMEOUT if it was set,
+ * ONNXB_ERR_CUDA if the stream reports an error, else ONNXB_OK.
+ */
+onnxb_status onnxb_last_device_status(void *cuda_stream);
+
+/*
+ * onnxb_set_kernel_override - force a kernel family for descriptors created
+ * afterwards (A/B measurements and tests): -1 = automatic choice (default),
+ * otherwise an onnxb_kernel_family value.  A forced family that cannot compute a
+ * given problem makes onnx_conv2d_desc return ERR_UNSUPPORTED.  Also settable
+ * through the environment variable ONNXB_FORCE = simt | mma | auto, read once.
+ */
+void onnxb_set_kernel_override(int family);
+
+/* Number of kernels this library has launched since it was loaded (all streams). */
+uint64_t onnxb_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ONNX_B200_H_ */

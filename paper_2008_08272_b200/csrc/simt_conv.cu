@@ -1,0 +1,191 @@
+// SIMT (fp32 FMA) convolution kernels: the path for contractions too thin for
+// the tensor cores (few input channels per group, depthwise) and the general
+// fallback that accepts every attribute combination of ONNX Conv (Sec. 4.1).
+#include <cuda_runtime.h>
+
+#include "common.h"
+
+namespace onnxb {
+
+namespace {
+
+constexpr int kDirectThreads = 128;   // one output pixel per thread
+constexpr int kDirectChunk = 256;     // reduction terms staged in shared memory per pass
+
+// Direct convolution.  A block owns 128 consecutive output pixels of one image
+// and MT consecutive output channels of one group; each thread keeps MT
+// accumulators, so every input value loaded is used MT times.  The reduction
+// index k = (c*kH + r)*kW + s is walked in chunks whose weights sit in shared
+// memory (all threads read the same weight: a broadcast).
+template <int MT>
+__global__ void __launch_bounds__(kDirectThreads)
+conv2d_direct_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
+                     const float *__restrict__ B, float *__restrict__ Y, int pixel_tiles, int m_tiles_per_group) {
+    __shared__ float wsm[MT * kDirectChunk];
+
+    const int tile = blockIdx.x % pixel_tiles;
+    const int n = blockIdx.x / pixel_tiles;
+    const int PQ = g.P * g.Q;
+    const int pix = tile * kDirectThreads + threadIdx.x;
+    const bool live = pix < PQ;
+    const int p = live ? pix / g.Q : 0;
+    const int q = live ? pix % g.Q : 0;
+    const int ih0 = p * g.sh - g.pt;
+    const int iw0 = q * g.sw - g.pl;
+    const int taps = g.kH * g.kW;
+    const int Kred = g.Cg * taps;
+
+    for (int mt = blockIdx.y; mt < m_tiles_per_group * g.group; mt += gridDim.y) {
+        const int grp = mt / m_tiles_per_group;
+        const int m0 = grp * g.Mg + (mt % m_tiles_per_group) * MT;
+        const int m_end = (grp + 1) * g.Mg;
+        const float *xg = X + ((size_t)n * g.C + (size_t)grp * g.Cg) * g.H * g.W;
+
+        float acc[MT];
+#pragma unroll
+        for (int j = 0; j < MT; ++j) acc[j] = 0.f;
+
+        for (int k0 = 0; k0 < Kred; k0 += kDirectChunk) {
+            const int len = min(kDirectChunk, Kred - k0);
+            __syncthreads();
+            for (int idx = threadIdx.x; idx < MT * len; idx += kDirectThreads) {
+                const int j = idx / len, kk = idx - j * len;
+                wsm[j * kDirectChunk + kk] = (m0 + j < m_end) ? W[(size_t)(m0 + j) * Kred + k0 + kk] : 0.f;
+            }
+            __syncthreads();
+            if (live) {
+                int c = k0 / taps;
+                int rs = k0 - c * taps;
+                int r = rs / g.kW;
+                int s = rs - r * g.kW;
+                for (int kk = 0; kk < len; ++kk) {
+                    const int ih = ih0 + r * g.dh;
+                    const int iw = iw0 + s * g.dw;
+                    float x = 0.f;
+                    if ((unsigned)ih < (unsigned)g.H && (unsigned)iw < (unsigned)g.W)
+                        x = __ldg(xg + ((size_t)c * g.H + ih) * g.W + iw);
+#pragma unroll
+                    for (int j = 0; j < MT; ++j) acc[j] = fmaf(x, wsm[j * kDirectChunk + kk], acc[j]);
+                    if (++s == g.kW) {
+                        s = 0;
+                        if (++r == g.kH) {
+                            r = 0;
+                            ++c;
+                        }
+                    }
+                }
+            }
+        }
+        if (live) {
+#pragma unroll
+            for (int j = 0; j < MT; ++j) {
+                const int m = m0 + j;
+                if (m < m_end) {
+                    float v = acc[j] + (B ? __ldg(B + m) : 0.f);
+                    if (g.relu) v = v > 0.f ? v : 0.f;
+                    Y[((size_t)n * g.M + m) * PQ + pix] = v;
+                }
+            }
+        }
+    }
+}
+
+// Depthwise convolution (group == C == M): purely HBM-bound, 2*kH*kW flops per
+// output.  A block stages the input window of a TP x TQ output tile of one
+// (image, channel) plane in shared memory with coalesced row loads (zeros
+// outside the image), then every thread produces one output from shared memory.
+constexpr int kDwTP = 8, kDwTQ = 32;
+
+__global__ void __launch_bounds__(kDwTP *kDwTQ)
+conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
+                        const float *__restrict__ B, float *__restrict__ Y, int q_tiles, int p_tiles,
+                        int in_rows, int in_cols) {
+    extern __shared__ float tile[];           // [in_rows][in_cols] then weights [kH*kW]
+    float *wsm = tile + in_rows * in_cols;
+
+    int bid = blockIdx.x;
+    const int qt = bid % q_tiles; bid /= q_tiles;
+    const int pt_ = bid % p_tiles; bid /= p_tiles;
+    const int plane = bid;                    // n * C + c
+    const int c = plane % g.C;
+    const int p0 = pt_ * kDwTP, q0 = qt * kDwTQ;
+    const int ih0 = p0 * g.sh - g.pt, iw0 = q0 * g.sw - g.pl;
+    const float *xp = X + (size_t)plane * g.H * g.W;
+
+    const int taps = g.kH * g.kW;
+    for (int i = threadIdx.x; i < taps; i += blockDim.x) wsm[i] = W[(size_t)c * taps + i];
+    for (int i = threadIdx.x; i < in_rows * in_cols; i += blockDim.x) {
+        const int rr = i / in_cols, cc = i - rr * in_cols;
+        const int ih = ih0 + rr, iw = iw0 + cc;
+        float v = 0.f;
+        if ((unsigned)ih < (unsigned)g.H && (unsigned)iw < (unsigned)g.W) v = __ldg(xp + (size_t)ih * g.W + iw);
+        tile[i] = v;
+    }
+    __syncthreads();
+
+    const int tq = threadIdx.x % kDwTQ, tp = threadIdx.x / kDwTQ;
+    const int p = p0 + tp, q = q0 + tq;
+    if (p < g.P && q < g.Q) {
+        float acc = 0.f;
+        for (int r = 0; r < g.kH; ++r) {
+            const float *row = tile + (tp * g.sh + r * g.dh) * in_cols + tq * g.sw;
+            for (int s = 0; s < g.kW; ++s) acc = fmaf(row[s * g.dw], wsm[r * g.kW + s], acc);
+        }
+        acc += B ? __ldg(B + c) : 0.f;
+        if (g.relu) acc = acc > 0.f ? acc : 0.f;
+        Y[((size_t)plane * g.P + p) * g.Q + q] = acc;
+    }
+}
+
+void depthwise_window(const ConvGeom &g, int &rows, int &cols) {
+    rows = (kDwTP - 1) * g.sh + (g.kH - 1) * g.dh + 1;
+    cols = (kDwTQ - 1) * g.sw + (g.kW - 1) * g.dw + 1;
+}
+
+}  // namespace
+
+bool simt_depthwise_supports(const ConvGeom &g) {
+    if (!(g.Cg == 1 && g.Mg == 1)) return false;
+    int rows, cols;
+    depthwise_window(g, rows, cols);
+    const long long floats = (long long)rows * cols + (long long)g.kH * g.kW;
+    if (floats * 4 > 40 * 1024) return false;
+    const long long q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;
+    return q_tiles * p_tiles * (long long)g.N * g.C <= 2147483647LL;
+}
+
+int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+                          void *stream) {
+    int rows, cols;
+    depthwise_window(g, rows, cols);
+    const int q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;
+    const size_t smem = ((size_t)rows * cols + (size_t)g.kH * g.kW) * sizeof(float);
+    const unsigned blocks = (unsigned)((long long)q_tiles * p_tiles * g.N * g.C);
+    conv2d_depthwise_kernel<<<blocks, kDwTP * kDwTQ, smem, (cudaStream_t)stream>>>(g, X, W, B, Y, q_tiles, p_tiles,
+                                                                                 rows, cols);
+    count_launch();
+    return (int)cudaGetLastError();
+}
+
+int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+                     void *stream) {
+    const long long PQ = (long long)g.P * g.Q;
+    const int pixel_tiles = (int)((PQ + kDirectThreads - 1) / kDirectThreads);
+    const long long gx = (long long)pixel_tiles * g.N;
+    if (gx > 2147483647LL) return (int)cudaErrorInvalidConfiguration;
+    const int MT = g.Mg >= 8 ? 8 : (g.Mg >= 4 ? 4 : 1);
+    const int m_tiles_per_group = (g.Mg + MT - 1) / MT;
+    const long long m_tiles = (long long)m_tiles_per_group * g.group;
+    dim3 grid((unsigned)gx, (unsigned)(m_tiles > 65535 ? 65535 : m_tiles), 1);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (MT == 8)
+        conv2d_direct_kernel<8><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+    else if (MT == 4)
+        conv2d_direct_kernel<4><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+    else
+        conv2d_direct_kernel<1><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+    count_launch();
+    return (int)cudaGetLastError();
+}
+
+}  // namespace onnxb

@@ -1,0 +1,254 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.  Bar: |gpu - oracle| <= 1e-3 * sum|x*w| + 1e-5 per
+output element; output shapes, index mapping and integer-valued cases bit-exact."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2008_08272_b200 import workloads as wl
+
+from parity import check_conv, run_conv_gpu, run_gemm_gpu, worst_ratio
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2008_08272_b200 import binding as b
+    b.load(build_if_missing=False)      # the compiled library must be there: no fallback
+    return b
+
+
+with open(os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")) as fh:
+    HAND = json.load(fh)
+
+
+@pytest.mark.parametrize("case", HAND["conv"], ids=lambda c: c["name"])
+def test_conv_hand_cases_bit_exact(binding, case):
+    X = np.array(case["x"], np.float32).reshape(case["x_shape"])
+    W = np.array(case["w"], np.float32).reshape(case["w_shape"])
+    B = np.array(case["b"], np.float32) if "b" in case else None
+    got, _ = run_conv_gpu(binding, torch, X, W, B, pads=case.get("pads", (0, 0, 0, 0)),
+                          strides=case.get("strides", (1, 1)), dilations=case.get("dilations", (1, 1)),
+                          group=case.get("group", 1), relu=case.get("relu", False))
+    assert list(got.shape) == case["y_shape"]
+    assert np.array_equal(got.ravel().astype(np.float64), np.array(case["y"], np.float64))
+
+
+@pytest.mark.parametrize("case", HAND["gemm"], ids=lambda c: c["name"])
+def test_gemm_hand_cases_bit_exact(binding, case):
+    A = np.array(case["a"], np.float32).reshape(case["a_shape"])
+    B = np.array(case["b"], np.float32).reshape(case["b_shape"])
+    C = np.array(case["c"], np.float32).reshape(case["c_shape"]) if "c" in case else None
+    got = run_gemm_gpu(binding, torch, A, B, C, alpha=case.get("alpha", 1.0), beta=case.get("beta", 1.0),
+                       transA=case.get("transA", False), transB=case.get("transB", False),
+                       fuse_relu=case.get("relu", False))
+    assert np.array_equal(got.ravel().astype(np.float64), np.array(case["y"], np.float64))
+
+
+def _random_conv_problems(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        g = int(rng.choice([1, 1, 1, 2, 3, 4]))
+        Cg, Mg = int(rng.integers(1, 9)), int(rng.integers(1, 11))
+        H, W = int(rng.integers(1, 24)), int(rng.integers(1, 24))
+        kH, kW = int(rng.integers(1, 6)), int(rng.integers(1, 6))
+        sh, sw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        dh, dw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        pads = tuple(int(v) for v in rng.integers(0, 4, 4))
+        if H + pads[0] + pads[2] < (kH - 1) * dh + 1 or W + pads[1] + pads[3] < (kW - 1) * dw + 1:
+            continue
+        out.append(dict(N=int(rng.integers(1, 4)), C=Cg * g, M=Mg * g, Cg=Cg, H=H, W=W, kH=kH, kW=kW,
+                        strides=(sh, sw), dilations=(dh, dw), pads=pads, group=g,
+                        bias=bool(rng.integers(0, 2)), relu=bool(rng.integers(0, 2)), seed=int(rng.integers(1 << 30))))
+    return out
+
+
+@pytest.mark.parametrize("p", _random_conv_problems(60, 1234), ids=lambda p: "x".join(
+    str(p[k]) for k in ("N", "C", "H", "W", "M", "kH", "kW", "group")))
+def test_conv_random_small(binding, p):
+    rng = np.random.default_rng(p["seed"])
+    X = rng.standard_normal((p["N"], p["C"], p["H"], p["W"])).astype(np.float32)
+    W = rng.standard_normal((p["M"], p["Cg"], p["kH"], p["kW"])).astype(np.float32)
+    B = rng.standard_normal((p["M"],)).astype(np.float32) if p["bias"] else None
+    ratio, _ = check_conv(binding, torch, X, W, B, relu=p["relu"], pads=p["pads"], strides=p["strides"],
+                          dilations=p["dilations"], group=p["group"])
+    assert ratio <= 1.0, ratio
+
+
+# shapes that span several tiles of every kernel family and leave ragged tails
+MID_CASES = [
+    dict(x=(2, 32, 30, 30), w=(48, 32, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(3, 64, 17, 19), w=(96, 64, 1, 1)),
+    dict(x=(2, 40, 29, 31), w=(72, 40, 1, 1), strides=(2, 2)),
+    dict(x=(2, 24, 33, 35), w=(40, 24, 3, 3), pads=(1, 1, 1, 1), strides=(2, 2)),
+    dict(x=(1, 16, 41, 37), w=(24, 16, 3, 3), pads=(2, 2, 2, 2), dilations=(2, 2)),
+    dict(x=(2, 3, 67, 65), w=(32, 3, 7, 7), pads=(3, 3, 3, 3), strides=(2, 2)),
+    dict(x=(2, 64, 20, 20), w=(64, 16, 3, 3), pads=(1, 1, 1, 1), group=4),
+    dict(x=(2, 96, 27, 29), w=(96, 1, 3, 3), pads=(1, 1, 1, 1), group=96),
+    dict(x=(2, 40, 31, 33), w=(40, 1, 5, 5), pads=(2, 2, 2, 2), strides=(2, 2), group=40),
+    dict(x=(1, 128, 7, 7), w=(256, 128, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(2, 256, 14, 14), w=(128, 256, 1, 1)),
+    dict(x=(1, 8, 9, 300), w=(16, 8, 1, 5), pads=(0, 2, 0, 2)),
+    dict(x=(1, 8, 300, 9), w=(16, 8, 5, 1), pads=(2, 0, 2, 0)),
+]
+
+
+@pytest.mark.parametrize("c", MID_CASES, ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+@pytest.mark.parametrize("relu", [False, True])
+def test_conv_multi_tile(binding, c, relu):
+    rng = np.random.default_rng(77)
+    X = rng.random(c["x"], dtype=np.float32)
+    fan = c["w"][1] * c["w"][2] * c["w"][3]
+    W = (rng.standard_normal(c["w"]) * np.sqrt(2.0 / fan)).astype(np.float32)
+    B = (rng.standard_normal((c["w"][0],)) * 0.1).astype(np.float32)
+    ratio, _ = check_conv(binding, torch, X, W, B, relu=relu, pads=c.get("pads", (0, 0, 0, 0)),
+                          strides=c.get("strides", (1, 1)), dilations=c.get("dilations", (1, 1)),
+                          group=c.get("group", 1))
+    assert ratio <= 1.0, ratio
+
+
+def test_conv_auto_pad_and_no_bias(binding):
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((2, 6, 13, 11)).astype(np.float32)
+    W = rng.standard_normal((4, 6, 4, 3)).astype(np.float32)
+    for mode in ("SAME_UPPER", "SAME_LOWER", "VALID"):
+        got, _ = run_conv_gpu(binding, torch, X, W, None, strides=(2, 3), auto_pad=mode)
+        want, S = oracle.conv2d(X, W, None, strides=(2, 3), auto_pad=mode)
+        assert worst_ratio(got, want, S) <= 1.0
+
+
+def test_delta_kernel_index_mapping_bit_exact(binding):
+    """A one-hot kernel turns Conv into a strided, shifted copy of one input channel.
+    With integer codes |v| <= 2048 (exact in TF32 and fp32) the result must be bit-exact."""
+    rng = np.random.default_rng(11)
+    N, C, H, W = 3, 20, 37, 41
+    X = rng.integers(-2048, 2049, size=(N, C, H, W)).astype(np.float32)
+    for (M, k, s, d, pad, g) in [(8, 3, 1, 1, 1, 1), (12, 3, 2, 1, 1, 1), (4, 5, 1, 2, 4, 1), (20, 3, 1, 1, 1, 20),
+                                 (10, 1, 2, 1, 0, 1), (40, 3, 1, 1, 1, 5)]:
+        Cg = C // g
+        Wt = np.zeros((M, Cg, k, k), np.float32)
+        for m in range(M):
+            Wt[m, (3 * m + 1) % Cg, (m + 1) % k, (2 * m) % k] = 1.0
+        got, _ = run_conv_gpu(binding, torch, X, Wt, None, pads=(pad,) * 4, strides=(s, s), dilations=(d, d), group=g)
+        want, _ = oracle.conv2d(X, Wt, None, pads=(pad,) * 4, strides=(s, s), dilations=(d, d), group=g, want_s=False)
+        assert np.array_equal(got.astype(np.float64), want)
+
+
+GEMM_CASES = [
+    # M, N, K, transA, transB, c_shape, alpha, beta, relu
+    (1, 1, 1, False, False, None, 1.0, 1.0, False),
+    (5, 7, 3, False, False, (), 1.0, 1.0, False),
+    (64, 10, 256, False, True, (10,), 1.0, 1.0, False),
+    (65, 130, 70, True, False, (1, 130), 0.5, -2.0, True),
+    (129, 67, 257, True, True, (129, 1), -1.5, 0.25, False),
+    (200, 136, 96, False, True, (200, 136), 1.0, 1.0, True),
+    (256, 384, 512, False, False, (384,), 1.0, 0.0, False),
+    (300, 300, 64, False, True, (300,), 2.0, 1.0, False),
+    (128, 1000, 2048, False, True, (1000,), 1.0, 1.0, False),
+    (96, 40, 1030, True, False, (1,), 1.0, 3.0, False),
+]
+
+
+@pytest.mark.parametrize("c", GEMM_CASES, ids=lambda c: f"{c[0]}x{c[1]}x{c[2]}_{int(c[3])}{int(c[4])}")
+def test_gemm_cases(binding, c):
+    M, N, K, tA, tB, cshape, alpha, beta, relu = c
+    rng = np.random.default_rng(M * 1000003 + N * 1009 + K)
+    A = rng.standard_normal((K, M) if tA else (M, K)).astype(np.float32)
+    B = rng.standard_normal((N, K) if tB else (K, N)).astype(np.float32)
+    C = rng.standard_normal(cshape).astype(np.float32) if cshape is not None else None
+    got = run_gemm_gpu(binding, torch, A, B, C, alpha=alpha, beta=beta, transA=tA, transB=tB, fuse_relu=relu)
+    want, S = oracle.gemm(A, B, C, alpha=alpha, beta=beta, transA=tA, transB=tB, relu=relu)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
+# ----------------------------------------------------------------- the five configurations
+def test_config1_mnist_conv(binding):
+    case = wl.config1_mnist_conv()
+    X, W, B = wl.conv_inputs(case)
+    ratio, fam = check_conv(binding, torch, X, W, B, relu=case.relu, **_kw(case))
+    assert ratio <= 1.0, (ratio, fam)
+
+
+def test_config2_gemm_head(binding):
+    case = wl.config2_gemm_head()
+    A, B, C = wl.gemm_inputs(case)
+    got = run_gemm_gpu(binding, torch, A, B, C, alpha=case.alpha, beta=case.beta, transA=case.transA,
+                       transB=case.transB, fuse_relu=case.relu)
+    want, S = oracle.gemm(A, B, C, alpha=case.alpha, beta=case.beta, transA=case.transA, transB=case.transB,
+                          relu=case.relu)
+    assert got.shape == (64, 10)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
+def _kw(case):
+    return dict(pads=case.pads, strides=case.strides, dilations=case.dilations, group=case.group)
+
+
+def test_config3_stage2_3x3_full_tensor(binding):
+    case = wl.config3_stage2_3x3()
+    X, W, B = wl.conv_inputs(case)
+    ratio, fam = check_conv(binding, torch, X, W, B, relu=case.relu, **_kw(case))
+    assert ratio <= 1.0, (ratio, fam)
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config4_stem_and_projection_full_tensor(binding, idx):
+    case = wl.config4_stem_and_projection()[idx]
+    X, W, B = wl.conv_inputs(case)
+    ratio, fam = check_conv(binding, torch, X, W, B, relu=case.relu, **_kw(case))
+    assert ratio <= 1.0, (ratio, fam)
+
+
+def _unique_sweep_cases():
+    seen, out = set(), []
+    for c in wl.resnet50_v1_convs():
+        key = (c.x_shape, c.w_shape, c.strides)
+        if key not in seen:
+            seen.add(key)
+            out.append(c)
+    return out + [wl.config5_depthwise()]
+
+
+@pytest.mark.parametrize("case", _unique_sweep_cases(), ids=lambda c: c.name)
+def test_config5_sweep_batch64_sampled_images(binding, case):
+    """Full batch-64 launch (the configuration the benchmark times); the oracle checks
+    images 0, 21, 42, 63 exactly (an image's outputs depend on that image only)."""
+    X, W, B = wl.conv_inputs(case)
+    ratio, fam = check_conv(binding, torch, X, W, B, relu=case.relu, images=[0, 21, 42, 63], **_kw(case))
+    assert ratio <= 1.0, (ratio, fam)
+
+
+def test_sweep_index_mapping_on_full_batch(binding):
+    """Delta kernels on full batch-64 tensors of three sweep shapes: bit-exact copy semantics
+    pin the index mapping of every image, not only the sampled ones."""
+    rng = np.random.default_rng(99)
+    for (C, HW, M, k, s, p) in [(64, 56, 64, 3, 1, 1), (256, 56, 128, 1, 2, 0), (512, 7, 512, 3, 1, 1)]:
+        X = rng.integers(-1024, 1025, size=(64, C, HW, HW)).astype(np.float32)
+        Wt = np.zeros((M, C, k, k), np.float32)
+        sel = [((5 * m + 3) % C, (m + 1) % k, (m // 2) % k) for m in range(M)]
+        for m, (c, r, t) in enumerate(sel):
+            Wt[m, c, r, t] = 1.0
+        got, _ = run_conv_gpu(binding, torch, X, Wt, None, pads=(p,) * 4, strides=(s, s))
+        Xp = np.zeros((64, C, HW + 2 * p, HW + 2 * p), np.float32)
+        Xp[:, :, p:p + HW, p:p + HW] = X
+        P = got.shape[2]
+        for m in range(0, M, 7):
+            c, r, t = sel[m]
+            want = Xp[:, c, r:r + (P - 1) * s + 1:s, t:t + (P - 1) * s + 1:s]
+            assert np.array_equal(got[:, m], want), (C, HW, m)
+
+
+def test_run_rejects_short_workspace_and_host_tensors(binding):
+    x = torch.zeros((1, 4, 8, 8), device="cuda")
+    w = torch.zeros((4, 4, 3, 3), device="cuda")
+    with pytest.raises(TypeError):
+        binding.onnx_conv2d(x.cpu(), w)
+    y = binding.onnx_conv2d(x, w)
+    assert y.shape == (1, 4, 6, 6) and float(y.abs().max()) == 0.0
