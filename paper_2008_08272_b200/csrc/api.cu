@@ -3,12 +3,48 @@
 #include <cuda_runtime.h>
 
 #include "common.h"
+#include "tc_host.h"
 
 using namespace onnxb;
 
 namespace onnxb {
 // Error word set by bounded device-side waits that ran out.
 __device__ unsigned int g_device_status_word = 0;
+unsigned int *device_status_ptr() {
+    static unsigned int *ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status_word) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<unsigned int *>(p);
+    }
+    return ptrs[dev];
+}
+
+// A 1x1, stride-1, unpadded, ungrouped convolution is one GEMM per image:
+// Y[n] (M x HW) = W (M x C) * X[n] (C x HW), with W K-major and X[n] pixel-major.
+static TcGemmProblem conv1x1_as_gemm(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y) {
+    TcGemmProblem t{};
+    const long long HW = (long long)g.H * g.W;
+    t.M = g.M; t.N = (int)HW; t.K = g.C; t.batch = g.N;
+    t.A = W; t.B = X;
+    t.a_mn_major = 0; t.b_mn_major = 1;
+    t.a_ld = g.C; t.b_ld = HW; t.a_bs = 0; t.b_bs = (long long)g.C * HW;
+    t.a_batched = 0; t.b_batched = 1;
+    t.alpha = 1.f; t.beta = 0.f; t.C = nullptr;
+    t.row_bias = B; t.relu = g.relu;
+    t.Y = Y; t.y_ld = HW; t.y_bs = (long long)g.M * HW;
+    return t;
+}
+
+bool conv_fits_mma_gemm(const ConvGeom &g) {
+    if (!(g.kH == 1 && g.kW == 1 && g.sh == 1 && g.sw == 1 && g.group == 1)) return false;
+    if (g.pt || g.pl || g.pb || g.pr) return false;
+    if (g.C < 32) return false;              // thin contraction: exact fp32 FMA instead
+    return tc_gemm_supports(conv1x1_as_gemm(g, nullptr, nullptr, nullptr, nullptr));
+}
+
 }  // namespace onnxb
 
 static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
@@ -29,6 +65,9 @@ extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, c
             break;
         case ONNXB_KERNEL_SIMT_DIRECT:
             err = launch_simt_conv(d->g, X, W, B, Y, cuda_stream);
+            break;
+        case ONNXB_KERNEL_MMA_GEMM:
+            err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y), cuda_stream);
             break;
         default:
             return ONNXB_ERR_UNSUPPORTED;
@@ -66,7 +105,22 @@ extern "C" onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float
     if (misaligned(A) || misaligned(B) || misaligned(C) || misaligned(Y) || misaligned(workspace))
         return ONNXB_ERR_UNSUPPORTED;
 
-    const int err = launch_simt_gemm(p, A, B, C, Y, cuda_stream);
+    // Tensor-core path unless the contraction is thin or an operand cannot be described to TMA.
+    TcGemmProblem t{};
+    t.M = p.M; t.N = p.N; t.K = p.K; t.batch = 1;
+    t.A = A; t.B = B;
+    t.a_mn_major = p.transA; t.a_ld = p.transA ? p.M : p.K;
+    t.b_mn_major = !p.transB; t.b_ld = p.transB ? p.K : p.N;
+    t.alpha = alpha; t.beta = beta; t.C = C; t.c_si = p.c_stride_i; t.c_sj = p.c_stride_j; t.c_sb = 0;
+    t.row_bias = nullptr; t.relu = p.relu;
+    t.Y = Y; t.y_ld = p.N; t.y_bs = 0;
+    const int forced = kernel_override();
+    const bool want_tc = forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT ||
+                         (forced < 0 && p.K >= 32);
+    int err;
+    if (want_tc && tc_gemm_supports(t)) err = launch_tc_gemm(t, cuda_stream);
+    else if (forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT) return ONNXB_ERR_UNSUPPORTED;
+    else err = launch_simt_gemm(p, A, B, C, Y, cuda_stream);
     return err == 0 ? ONNXB_OK : ONNXB_ERR_CUDA;
 }
 

@@ -42,6 +42,7 @@ int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const fl
 int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
                           void *stream);
 bool simt_depthwise_supports(const ConvGeom &g);
+bool conv_fits_mma_gemm(const ConvGeom &g);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
 
 struct GemmProblem {
     int M, N, K;

@@ -130,11 +130,15 @@ extern "C" onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *a, onnxb_conv
     const int forced = kernel_override();
     int family = ONNXB_KERNEL_SIMT_DIRECT;
     if (simt_depthwise_supports(g)) family = ONNXB_KERNEL_SIMT_DEPTHWISE;
+    else if (conv_fits_mma_gemm(g)) family = ONNXB_KERNEL_MMA_GEMM;
     if (forced == ONNXB_KERNEL_SIMT_DIRECT) family = ONNXB_KERNEL_SIMT_DIRECT;
     else if (forced == ONNXB_KERNEL_SIMT_DEPTHWISE) {
         if (!simt_depthwise_supports(g)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
         family = ONNXB_KERNEL_SIMT_DEPTHWISE;
-    } else if (forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT) {
+    } else if (forced == ONNXB_KERNEL_MMA_GEMM) {
+        if (!conv_fits_mma_gemm(g)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
+        family = ONNXB_KERNEL_MMA_GEMM;
+    } else if (forced == ONNXB_KERNEL_MMA_IMPLICIT) {
         delete d;
         return ONNXB_ERR_UNSUPPORTED;
     }

@@ -1,0 +1,393 @@
+// Batched TF32 GEMM on the 5th-generation tensor cores:
+//     D[b] (M x N) = A'[b] (M x K) * B'[b] (K x N),   then a fused epilogue.
+//
+// It serves ONNX Gemm (Sec. 3.4.3) and every 1x1, stride-1 convolution (Sec. 4.1),
+// which in NCHW is one GEMM per image: Y[n] (Cout x HW) = W (Cout x C) * X[n] (C x HW).
+//
+// Pipeline (one persistent CTA per SM, 192 threads):
+//   warp 0    TMA producer: fp32 operand tiles, 128-byte swizzled, into a ring of
+//             shared-memory stages, completion signalled on mbarriers;
+//   warp 1    one thread issues tcgen05.mma kind::tf32 (128 x BN x 8 per instruction) into
+//             one of two TMEM accumulators and commits stage releases to mbarriers;
+//   warps 2-5 epilogue: tcgen05.ld the finished accumulator (while the MMA warp fills the
+//             other one), apply alpha / beta*C / bias / Relu, stage 32x32 blocks in swizzled
+//             shared memory and write them with TMA stores (plain stores when Y cannot be
+//             described by a tensor map).
+// Either operand may be K-major (reduction index contiguous) or MN-major (row/column
+// index contiguous, e.g. the pixels of an NCHW image); no transposed copy is ever made.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "common.h"
+#include "tc_common.cuh"
+#include "tc_host.h"
+
+namespace onnxb {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kBM = 128;            // UMMA M: rows of D per tile (TMEM lanes)
+constexpr int kBK = 32;             // fp32 elements per stage along K (one 128-byte swizzle row)
+constexpr int kMaxBN = 256;         // UMMA N limit
+constexpr int kMaxStages = 8;
+constexpr int kThreads = 192;
+constexpr int kABytes = kBM * kBK * 4;             // 16 KB
+constexpr int kStoreBufBytes = 32 * 32 * 4;        // one 32x32 fp32 block
+constexpr int kStagingBytes = 4 * 2 * kStoreBufBytes;
+constexpr int kBarrierBytes = 256;
+constexpr int kSmemLimit = 232448;                 // 227 KB opt-in maximum per CTA
+
+struct Params {
+    int M, N, K, batch;
+    int a_mn, b_mn;            // operand is MN-major (else K-major)
+    int a_batched, b_batched;
+    int BN, tiles_m, tiles_n, num_kb, num_stages;
+    uint32_t idesc, stage_bytes, tx_bytes;
+    float alpha, beta;
+    const float *C;            // optional addend, element strides below (0 = broadcast)
+    long long c_si, c_sj, c_sb;
+    const float *row_bias;     // optional per-row addend (convolution bias)
+    int relu;
+    float *Y;                  // used by the plain-store epilogue
+    long long y_ld, y_sb;
+    int y_tma;
+    unsigned int *err;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmY, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *stages = smem;
+    uint8_t *staging = smem + (size_t)p.num_stages * p.stage_bytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + kStagingBytes);
+    uint64_t *full = bars, *empty = bars + kMaxStages;
+    uint64_t *tmem_full = bars + 2 * kMaxStages, *tmem_empty = tmem_full + 2;
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tmem_empty + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.tiles_m * p.tiles_n * p.batch;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.num_stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&tmem_full[a], 1);
+            mbar_init(&tmem_empty[a], 4);
+        }
+        mbar_fence_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+        if (p.y_tma) prefetch_tmap(&tmY);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_holder, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+                const int tm = t % p.tiles_m;
+                const int tn = (t / p.tiles_m) % p.tiles_n;
+                const int b = t / (p.tiles_m * p.tiles_n);
+                const int ab = p.a_batched ? b : 0, bb = p.b_batched ? b : 0;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
+                    mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
+                    uint8_t *sA = stages + (size_t)stage * p.stage_bytes;
+                    uint8_t *sB = sA + kABytes;
+                    if (!p.a_mn) {
+                        tma_load_3d(sA, &tmA, &full[stage], kb * kBK, tm * kBM, ab);
+                    } else {
+                        for (int j = 0; j < kBM / 32; ++j)
+                            tma_load_3d(sA + j * 4096, &tmA, &full[stage], tm * kBM + j * 32, kb * kBK, ab);
+                    }
+                    if (!p.b_mn) {
+                        tma_load_3d(sB, &tmB, &full[stage], kb * kBK, tn * p.BN, bb);
+                    } else {
+                        for (int j = 0; j < p.BN / 32; ++j)
+                            tma_load_3d(sB + j * 4096, &tmB, &full[stage], tn * p.BN + j * 32, kb * kBK, bb);
+                    }
+                    if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+                mbar_wait(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * kMaxBN;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    mbar_wait(&full[stage], phase, p.err, 3);
+                    tc_fence_after_sync();
+                    const uint32_t sA = smem_u32(stages + (size_t)stage * p.stage_bytes);
+                    const uint32_t sB = sA + kABytes;
+                    const int k_left = p.K - kb * kBK;
+                    const int k8 = k_left >= kBK ? kBK / 8 : (k_left + 7) / 8;
+                    for (int k = 0; k < k8; ++k) {
+                        // K-major: 32 bytes further along the swizzled 128-byte rows (8-row groups
+                        // 1024 bytes apart).  MN-major 32-bit operands use the 128-byte swizzle with
+                        // 32-byte atoms: atoms of four 128-byte K rows (512 bytes apart along K), blocks
+                        // of 32 rows/columns 4096 bytes apart; one instruction consumes eight K rows.
+                        const uint64_t ad = p.a_mn ? make_smem_desc(sA + k * 1024, 4096, 512, kSwizzle128B32)
+                                                   : make_smem_desc(sA + k * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = p.b_mn ? make_smem_desc(sB + k * 1024, 4096, 512, kSwizzle128B32)
+                                                   : make_smem_desc(sB + k * 32, 16, 1024, kSwizzle128B);
+                        mma_tf32(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                    }
+                    mma_commit(&empty[stage]);
+                    if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+                }
+                mma_commit(&tmem_full[acc]);
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                    // TMEM lane quarter this warp may read
+        uint8_t *my_staging = staging + q * 2 * kStoreBufBytes;
+        int acc = 0;
+        uint32_t acc_phase = 0, store_idx = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            const int tm = t % p.tiles_m;
+            const int tn = (t / p.tiles_m) % p.tiles_n;
+            const int b = t / (p.tiles_m * p.tiles_n);
+            mbar_wait(&tmem_full[acc], acc_phase, p.err, 4);
+            tc_fence_after_sync();
+            const int row0 = tm * kBM + q * 32;
+            const int row = row0 + lane;
+            if (row0 < p.M) {
+                const float rb = (p.row_bias && row < p.M) ? __ldg(p.row_bias + row) : 0.f;
+                for (int chunk = 0; chunk < p.BN / 32; ++chunk) {
+                    const int col0 = tn * p.BN + chunk * 32;
+                    if (col0 >= p.N) break;
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBN + chunk * 32), v);
+                    tmem_ld_wait();
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float x = p.alpha * __uint_as_float(v[j]) + rb;
+                        if (p.C && row < p.M && col0 + j < p.N)
+                            x = fmaf(p.beta, __ldg(p.C + b * p.c_sb + row * p.c_si + (col0 + j) * p.c_sj), x);
+                        if (p.relu) x = x > 0.f ? x : 0.f;
+                        f[j] = x;
+                    }
+                    if (p.y_tma) {
+                        uint8_t *buf = my_staging + (store_idx & 1) * kStoreBufBytes;
+                        ++store_idx;
+                        if (lane == 0) tma_store_wait_read<1>();   // the store that last read this buffer is done
+                        __syncwarp();
+                        // row `lane` of the block, 16-byte chunk c stored at position c ^ (lane % 8)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            float4 val = make_float4(f[4 * c], f[4 * c + 1], f[4 * c + 2], f[4 * c + 3]);
+                            *reinterpret_cast<float4 *>(buf + lane * 128 + ((c ^ (lane & 7)) << 4)) = val;
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_3d(&tmY, buf, col0, row0, b);
+                            tma_store_commit();
+                        }
+                    } else if (row < p.M) {
+                        float *yrow = p.Y + b * p.y_sb + (long long)row * p.y_ld;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) yrow[col0 + j] = f[j];
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+            acc ^= 1;
+            if (acc == 0) acc_phase ^= 1;
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+int pick_bn(long long tiles_m, long long n, long long batch, int num_sms) {
+    if (n <= 32) return 32;
+    int best = 32;
+    double best_cost = 1e300;
+    for (int bn = 32; bn <= kMaxBN; bn += 32) {
+        const long long tiles = tiles_m * ((n + bn - 1) / bn) * batch;
+        const long long waves = (tiles + num_sms - 1) / num_sms;
+        const double cost = (double)waves * (bn + 48);
+        if (cost < best_cost - 1e-9 || (cost < best_cost + 1e-9 && bn > best)) {
+            best_cost = cost;
+            best = bn;
+        }
+    }
+    return best;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ host side
+namespace tc_host {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+bool make_tmap(CUtensorMap *out, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
+               const uint32_t *box, int swizzle) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[5], gstr[4];
+    cuuint32_t bdim[5], estr[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bdim[i] = box[i];
+        estr[i] = 1;
+        if (i > 0) gstr[i - 1] = strides_bytes[i - 1];
+    }
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void *>(base), gdim, gstr, bdim, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle == kTmapSwizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B
+              : swizzle == kTmapSwizzle128Atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B
+                                                 : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int num_sms() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            return 148;
+    }
+    return n;
+}
+
+}  // namespace tc_host
+
+bool tc_gemm_supports(const TcGemmProblem &g) {
+    if (g.M < 1 || g.N < 1 || g.K < 1 || g.batch < 1) return false;
+    // tensor-map strides must be multiples of 16 bytes
+    if (g.a_ld % 4 || g.b_ld % 4) return false;
+    if (g.batch > 1 && ((g.a_batched && g.a_bs % 4) || (g.b_batched && g.b_bs % 4))) return false;
+    if ((long long)((g.M + kBM - 1) / kBM) * g.batch > 0x7fffffffLL / 4096) return false;
+    return true;
+}
+
+int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
+    using namespace tc_host;
+    Params p{};
+    p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
+    p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
+    p.a_batched = g.a_batched && g.batch > 1; p.b_batched = g.b_batched && g.batch > 1;
+    p.tiles_m = (g.M + kBM - 1) / kBM;
+    const int sms = num_sms();
+    p.BN = pick_bn(p.tiles_m, g.N, g.batch, sms);
+    p.tiles_n = (g.N + p.BN - 1) / p.BN;
+    p.num_kb = (g.K + kBK - 1) / kBK;
+    p.stage_bytes = (uint32_t)(kABytes + p.BN * 128);
+    p.tx_bytes = p.stage_bytes;
+    int stages = (kSmemLimit - 1024 - kBarrierBytes - kStagingBytes) / (int)p.stage_bytes;
+    p.num_stages = stages > kMaxStages ? kMaxStages : stages;
+    p.idesc = tc::make_idesc_tf32(kBM, p.BN, p.a_mn, p.b_mn);
+    p.alpha = g.alpha; p.beta = g.beta;
+    p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
+    p.row_bias = g.row_bias; p.relu = g.relu;
+    p.Y = g.Y; p.y_ld = g.y_ld; p.y_sb = g.y_bs;
+    p.y_tma = (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);
+    p.err = device_status_ptr();
+    if (!p.err) return (int)cudaErrorUnknown;
+
+    CUtensorMap tmA, tmB, tmY;
+    // operand maps: dim0 is the contiguous axis
+    {
+        const uint64_t rows = (uint64_t)g.M, k = (uint64_t)g.K;
+        uint64_t dims[3], str[2];
+        uint32_t box[3];
+        if (!p.a_mn) { dims[0] = k; dims[1] = rows; box[0] = kBK; box[1] = kBM; }
+        else { dims[0] = rows; dims[1] = k; box[0] = 32; box[1] = kBK; }
+        dims[2] = p.a_batched ? (uint64_t)g.batch : 1;
+        box[2] = 1;
+        str[0] = (uint64_t)g.a_ld * 4;
+        str[1] = p.a_batched ? (uint64_t)g.a_bs * 4 : str[0] * dims[1];
+        if (!make_tmap(&tmA, g.A, 3, dims, str, box, p.a_mn ? kTmapSwizzle128Atom32 : kTmapSwizzle128))
+            return (int)cudaErrorInvalidValue;
+    }
+    {
+        const uint64_t cols = (uint64_t)g.N, k = (uint64_t)g.K;
+        uint64_t dims[3], str[2];
+        uint32_t box[3];
+        if (!p.b_mn) { dims[0] = k; dims[1] = cols; box[0] = kBK; box[1] = (uint32_t)p.BN; }
+        else { dims[0] = cols; dims[1] = k; box[0] = 32; box[1] = kBK; }
+        dims[2] = p.b_batched ? (uint64_t)g.batch : 1;
+        box[2] = 1;
+        str[0] = (uint64_t)g.b_ld * 4;
+        str[1] = p.b_batched ? (uint64_t)g.b_bs * 4 : str[0] * dims[1];
+        if (!make_tmap(&tmB, g.B, 3, dims, str, box, p.b_mn ? kTmapSwizzle128Atom32 : kTmapSwizzle128))
+            return (int)cudaErrorInvalidValue;
+    }
+    if (p.y_tma) {
+        uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.M, (uint64_t)g.batch};
+        uint64_t str[2] = {(uint64_t)g.y_ld * 4, g.batch > 1 ? (uint64_t)g.y_bs * 4 : (uint64_t)g.y_ld * 4 * g.M};
+        uint32_t box[3] = {32, 32, 1};
+        if (!make_tmap(&tmY, g.Y, 3, dims, str, box, kTmapSwizzle128)) return (int)cudaErrorInvalidValue;
+    } else {
+        tmY = tmA;   // never dereferenced
+    }
+
+    const size_t smem = 1024 + (size_t)p.num_stages * p.stage_bytes + kStagingBytes + kBarrierBytes;
+    const cudaError_t attr_err =
+        cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    if (attr_err != cudaSuccess) return (int)attr_err;
+    const long long total = (long long)p.tiles_m * p.tiles_n * p.batch;
+    const int grid = (int)(total < sms ? total : sms);
+    tc_gemm_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, tmY, p);
+    count_launch();
+    return (int)cudaGetLastError();
+}
+
+}  // namespace onnxb

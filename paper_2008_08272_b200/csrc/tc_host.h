@@ -1,0 +1,41 @@
+// Host-side interface of the tensor-core family.
+#pragma once
+#include <cuda.h>
+#include <cstdint>
+
+#include "common.h"
+
+namespace onnxb {
+
+// D[b] (M x N) = A'[b] (M x K) * B'[b] (K x N); Y = relu?(alpha*D + beta*C + row_bias).
+// An operand is "MN-major" when its row (A') / column (B') index is the contiguous one.
+// ld = element stride of the non-contiguous axis, bs = element stride between batches.
+struct TcGemmProblem {
+    int M, N, K, batch;
+    const float *A, *B;
+    int a_mn_major, b_mn_major;
+    long long a_ld, b_ld, a_bs, b_bs;
+    int a_batched, b_batched;
+    float alpha, beta;
+    const float *C;
+    long long c_si, c_sj, c_sb;
+    const float *row_bias;
+    int relu;
+    float *Y;
+    long long y_ld, y_bs;
+};
+
+bool tc_gemm_supports(const TcGemmProblem &g);
+int launch_tc_gemm(const TcGemmProblem &g, void *stream);
+
+// Address of the device error word of the current device (NULL on failure).
+unsigned int *device_status_ptr();
+
+namespace tc_host {
+constexpr int kTmapSwizzleNone = 0, kTmapSwizzle128 = 1, kTmapSwizzle128Atom32 = 2;
+bool make_tmap(CUtensorMap *out, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
+               const uint32_t *box, int swizzle);
+int num_sms();
+}  // namespace tc_host
+
+}  // namespace onnxb

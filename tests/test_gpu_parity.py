@@ -95,6 +95,9 @@ MID_CASES = [
     dict(x=(2, 40, 31, 33), w=(40, 1, 5, 5), pads=(2, 2, 2, 2), strides=(2, 2), group=40),
     dict(x=(1, 128, 7, 7), w=(256, 128, 3, 3), pads=(1, 1, 1, 1)),
     dict(x=(2, 256, 14, 14), w=(128, 256, 1, 1)),
+    dict(x=(2, 64, 56, 56), w=(256, 64, 1, 1)),
+    dict(x=(3, 96, 20, 20), w=(40, 96, 1, 1)),
+    dict(x=(2, 36, 12, 12), w=(130, 36, 1, 1)),
     dict(x=(1, 8, 9, 300), w=(16, 8, 1, 5), pads=(0, 2, 0, 2)),
     dict(x=(1, 8, 300, 9), w=(16, 8, 5, 1), pads=(2, 0, 2, 0)),
 ]
@@ -153,6 +156,11 @@ GEMM_CASES = [
     (300, 300, 64, False, True, (300,), 2.0, 1.0, False),
     (128, 1000, 2048, False, True, (1000,), 1.0, 1.0, False),
     (96, 40, 1030, True, False, (1,), 1.0, 3.0, False),
+    (256, 512, 128, True, False, (256, 512), 1.0, 1.0, True),
+    (384, 96, 200, True, True, (96,), 0.5, 1.0, False),
+    (100, 260, 36, False, False, None, 1.0, 1.0, False),
+    (128, 256, 32, False, True, None, 1.0, 1.0, False),
+    (1000, 2500, 520, False, True, (2500,), 1.0, 1.0, True),
 ]
 
 
