@@ -69,6 +69,9 @@ extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, c
         case ONNXB_KERNEL_MMA_GEMM:
             err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y), cuda_stream);
             break;
+        case ONNXB_KERNEL_MMA_IMPLICIT:
+            err = launch_tc_conv(d->plan, X, W, B, Y, workspace, cuda_stream);
+            break;
         default:
             return ONNXB_ERR_UNSUPPORTED;
     }

@@ -5,6 +5,7 @@
 #include <cstdint>
 
 #include "onnx_b200.h"
+#include "tc_conv_plan.h"
 
 namespace onnxb {
 
@@ -24,6 +25,7 @@ struct ConvGeom {
 struct onnxb_conv2d_desc_s {
     onnxb::ConvGeom g;
     int family;              // onnxb_kernel_family
+    onnxb::TcConvPlan plan;  // valid when family == ONNXB_KERNEL_MMA_IMPLICIT
     size_t workspace_bytes;
     int64_t y_dims[4];
     int64_t pads[4];
@@ -42,7 +44,12 @@ int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const fl
 int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
                           void *stream);
 bool simt_depthwise_supports(const ConvGeom &g);
-bool conv_fits_mma_gemm(const ConvGeom &g);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
+bool conv_fits_mma_gemm(const ConvGeom &g);
+// implicit-GEMM tensor-core convolution (tc_conv.cu)
+bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan);
+size_t tc_conv_workspace_bytes(const TcConvPlan &plan);
+int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, float *Y,
+                   void *workspace, void *stream);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
 
 struct GemmProblem {
     int M, N, K;

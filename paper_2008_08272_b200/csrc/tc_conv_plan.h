@@ -1,0 +1,102 @@
+// Geometry of the implicit-GEMM convolution kernel, shared by host planning and
+// device code (plain integer arithmetic, no CUDA types).
+//
+// "Slot space".  For every image the kernel lays the (zero-padded, stride-decimated)
+// input out as a grid of Hs x Ws slots per parity plane; slot (hq, wq) of plane (a, b)
+// holds the padded input pixel (hq*sh + a, wq*sw + b).  Output pixel (p, q) is anchored
+// at slot u = p*Ws + q, and filter tap (r, s) reads plane ((r*dh) % sh, (s*dw) % sw) at
+// slot u + ((r*dh)/sh)*Ws + (s*dw)/sw: a fixed shift per tap.  Images follow each other
+// every L = Hs*Ws slots, so a GEMM row tile is simply 128 consecutive global slots, and
+// the im2col operand of a tap is the same shared-memory tile read from a shifted start
+// address.  Hs and Ws are chosen as small as possible: the trailing zero padding of one
+// row (image) is allowed to alias the leading zero padding of the next.
+#pragma once
+#include <cstdint>
+
+#if defined(__CUDACC__)
+#define ONNXB_HD __host__ __device__
+#else
+#define ONNXB_HD
+#endif
+
+namespace onnxb {
+
+constexpr int kConvMaxPlanes = 4;
+constexpr int kConvMaxTaps = 64;
+constexpr int kConvMaxSeg = 8;
+constexpr int kConvKB = 16;            // input channels per pipeline step (four 16-byte chunks)
+
+struct TcConvPlan {
+    // problem
+    int N, C, H, W, M, Cg, Mg, kH, kW, P, Q, pt, pl, sh, sw, dh, dw, group, relu;
+    // slot space
+    int Hs, Ws, L;
+    long long total_slots;           // N * L
+    int planes, pa[kConvMaxPlanes], pb[kConvMaxPlanes];
+    int a_min, a_max;                // smallest / largest used row parity
+    int taps;
+    int tap_plane[kConvMaxTaps], tap_shift[kConvMaxTaps];
+    // tiling
+    int MT;                          // 128-row accumulator tiles per CTA tile (1 or 2)
+    int BN, ctiles;                  // output channels per tile, tiles per group
+    int SLOTS;                       // slots per plane held in one A stage = MT*128 + largest tap shift
+    int ncb;                         // channel blocks = ceil(Cg / kConvKB)
+    int pix_tiles;                   // ceil(total_slots / (MT*128))
+    long long total_tiles;
+    // raw staging
+    int raw_mode;                    // 0: tensor-map boxes [kConvKB][BOXP] over X seen as (H*W, N*C); 1: whole-image slabs
+    int BOXP;
+    // shared memory carve-up (bytes)
+    int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages;
+    int chunk_pitch, plane_pitch;    // bytes between 4-channel chunks / parity planes inside an A stage
+    uint32_t idesc;
+    long long packed_floats;         // size of the packed weight buffer
+};
+
+struct TcConvSegs {
+    int n_first, nseg;
+    int f0[kConvMaxSeg];             // first flat pixel (h*W + w) staged for the image
+    int base[kConvMaxSeg];           // float offset of the image's data inside the raw stage
+    int nbox[kConvMaxSeg];           // boxes (mode 0) / 1 (mode 1) / 0 when nothing of the image is needed
+    int total_floats;
+};
+
+// Which part of which images the A stage of the tile starting at global slot G0 needs.
+ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvSegs &t) {
+    long long Gend = G0 + g.SLOTS;
+    if (Gend > g.total_slots) Gend = g.total_slots;
+    t.n_first = (int)(G0 / g.L);
+    const int n_last = (int)((Gend - 1) / g.L);
+    t.nseg = n_last - t.n_first + 1;
+    if (t.nseg > kConvMaxSeg) t.nseg = kConvMaxSeg;   // excluded by the planner
+    int base = 0;
+    for (int i = 0; i < t.nseg; ++i) {
+        const long long n = t.n_first + i;
+        const long long lo = G0 > n * g.L ? G0 : n * g.L;
+        const long long hi = Gend < (n + 1) * g.L ? Gend : (n + 1) * g.L;
+        const int u_lo = (int)(lo - n * g.L), u_hi = (int)(hi - n * g.L);   // [u_lo, u_hi)
+        const int hq_lo = u_lo / g.Ws, hq_hi = (u_hi - 1) / g.Ws;
+        int h_min = hq_lo * g.sh + g.a_min - g.pt;
+        int h_max = hq_hi * g.sh + g.a_max - g.pt;
+        if (h_min < 0) h_min = 0;
+        if (h_max > g.H - 1) h_max = g.H - 1;
+        t.base[i] = base;
+        if (h_min > h_max) {
+            t.f0[i] = 0;
+            t.nbox[i] = 0;
+        } else if (g.raw_mode == 1) {
+            t.f0[i] = 0;
+            t.nbox[i] = 1;
+            base += kConvKB * g.H * g.W;
+        } else {
+            const int f0 = (h_min * g.W) & ~3;
+            const int len = (h_max + 1) * g.W - f0;
+            t.f0[i] = f0;
+            t.nbox[i] = (len + g.BOXP - 1) / g.BOXP;
+            base += t.nbox[i] * g.BOXP * kConvKB;
+        }
+    }
+    t.total_floats = base;
+}
+
+}  // namespace onnxb
