@@ -139,6 +139,34 @@ onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t desc, const float *X, const flo
 void onnx_conv2d_desc_destroy(onnxb_conv2d_desc_t desc);
 
 /*
+ * onnx_conv2d_run_static - the same computation as onnx_conv2d_run, for callers that
+ * cannot allocate device memory and therefore have no workspace to pass: a control loop
+ * whose memory budget was frozen at start-up, a plugin inside a host application that owns
+ * the allocator, a process whose device memory is already fully committed.  (This entry
+ * point is a convenience of this library; the paper has no counterpart.)
+ *
+ * The scratch comes from a fixed array of onnx_conv2d_static_scratch_bytes() bytes
+ * (10 MiB) that is part of the library image: every GPU the library is loaded on holds it
+ * until the process exits.  The call allocates and frees nothing.  A descriptor whose
+ * queried workspace_bytes exceeds that size is rejected with ONNXB_ERR_WORKSPACE and
+ * nothing is launched; use onnx_conv2d_run with your own workspace for such layers.
+ *
+ * X, W, B, Y, cuda_stream: exactly as for onnx_conv2d_run (device pointers, caller-owned).
+ * The first call on each device looks up the array's device address (a host-side query,
+ * not an allocation); make that first call outside any stream capture.
+ * All calls on a device share the one array, and it keeps whatever the previous call left
+ * there.  Each call overwrites all of the scratch it later reads, so stale contents are
+ * harmless, but two calls whose kernels may overlap on the GPU (different streams, or
+ * several host threads) race on it: serialise them, e.g. by using one stream.
+ * Errors: as onnx_conv2d_run, plus ONNXB_ERR_WORKSPACE as described above.
+ */
+onnxb_status onnx_conv2d_run_static(onnxb_conv2d_desc_t desc, const float *X, const float *W,
+                                    const float *B, float *Y, void *cuda_stream);
+
+/* Size in bytes of the built-in scratch array used by onnx_conv2d_run_static. */
+size_t onnx_conv2d_static_scratch_bytes(void);
+
+/*
  * onnx_gemm_workspace_bytes - device scratch onnx_gemm_run needs for this
  * problem (0 when none).  Host only.
  */

@@ -21,7 +21,8 @@ KERNEL_FAMILIES = ["simt_direct", "simt_depthwise", "mma_gemm", "mma_implicit"]
 
 EXPORTS = [
     "onnx_conv2d_desc", "onnx_conv2d_desc_query", "onnx_conv2d_desc_query_kernel", "onnx_conv2d_run",
-    "onnx_conv2d_desc_destroy", "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
+    "onnx_conv2d_desc_destroy", "onnx_conv2d_run_static", "onnx_conv2d_static_scratch_bytes",
+    "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
 ]
 
@@ -70,6 +71,10 @@ def load(build_if_missing: bool = True):
     lib.onnx_conv2d_desc_query_kernel.argtypes = [vp]
     lib.onnx_conv2d_run.restype = ctypes.c_int
     lib.onnx_conv2d_run.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.onnx_conv2d_run_static.restype = ctypes.c_int
+    lib.onnx_conv2d_run_static.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.onnx_conv2d_static_scratch_bytes.restype = sz
+    lib.onnx_conv2d_static_scratch_bytes.argtypes = []
     lib.onnx_conv2d_desc_destroy.restype = None
     lib.onnx_conv2d_desc_destroy.argtypes = [vp]
     lib.onnx_gemm_workspace_bytes.restype = sz
@@ -164,6 +169,18 @@ class Conv2dDesc:
                                          ws_ptr, ws_len, _stream_ptr(stream)), "onnx_conv2d_run")
         return Y
 
+    def run_static(self, X, W, B=None, Y=None, stream=None):
+        """``onnx_conv2d_run_static``: like run(), but the library's built-in scratch array
+        stands in for the workspace, so no device memory is allocated for scratch.  (Y is
+        still allocated here with torch when the caller does not pass one.)"""
+        import torch
+        if Y is None:
+            Y = torch.empty(self.y_shape, dtype=torch.float32, device=X.device)
+        _check(self._lib.onnx_conv2d_run_static(self._h, _dev_ptr(X, "X"), _dev_ptr(W, "W"),
+                                                _dev_ptr(B, "B", allow_none=True), _dev_ptr(Y, "Y"),
+                                                _stream_ptr(stream)), "onnx_conv2d_run_static")
+        return Y
+
     def close(self):
         if self._h:
             self._lib.onnx_conv2d_desc_destroy(self._h)
@@ -218,6 +235,10 @@ def onnx_gemm(A, B, C=None, *, alpha=1.0, beta=1.0, transA=False, transB=False, 
                              c_rank, c_dims, int(bool(fuse_relu)), _dev_ptr(Y, "Y"), ws_ptr, ws_len,
                              _stream_ptr(stream)), "onnx_gemm_run")
     return Y
+
+
+def static_scratch_bytes() -> int:
+    return int(load().onnx_conv2d_static_scratch_bytes())
 
 
 def last_device_status(stream=None) -> int:
