@@ -48,6 +48,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc] + NVCC_FLAGS + ["-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("ONNXB_NVCC_EXTRA", "").split()
     cmd += sources() + ["-o", tmp]
     proc = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if verbose or proc.returncode != 0:

@@ -46,7 +46,7 @@ int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, con
 bool simt_depthwise_supports(const ConvGeom &g);
 bool conv_fits_mma_gemm(const ConvGeom &g);
 // implicit-GEMM tensor-core convolution (tc_conv.cu)
-bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan);
+bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan, bool forced = false);
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan);
 int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, float *Y,
                    void *workspace, void *stream);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM

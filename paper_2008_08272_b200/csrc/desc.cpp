@@ -140,7 +140,7 @@ extern "C" onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *a, onnxb_conv
         if (!conv_fits_mma_gemm(g)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
         family = ONNXB_KERNEL_MMA_GEMM;
     } else if (forced == ONNXB_KERNEL_MMA_IMPLICIT) {
-        if (!tc_conv_plan(g, d->plan)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
+        if (!tc_conv_plan(g, d->plan, true)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
         family = ONNXB_KERNEL_MMA_IMPLICIT;
     }
     d->family = family;

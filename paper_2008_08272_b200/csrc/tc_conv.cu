@@ -1,14 +1,14 @@
 // Implicit-GEMM convolution on the tcgen05 tensor cores (TF32 multiply, fp32 accumulate)
-// for ONNX Conv (Sec. 4.1) with any kernel size, stride, dilation, padding and (wide) groups.
+// for ONNX Conv (Sec. 4.1) with any kernel size, stride, dilation, padding and groups.
 //
 // GEMM view: rows = output pixels ("anchors" in slot space, see tc_conv_plan.h), columns =
 // output channels, reduction = input channels x filter taps.  The im2col matrix is never
-// formed; per block of 16 input channels
+// formed; per block of KB input channels
 //   warp 0      stages the raw NCHW rows the tile touches into shared memory by TMA
 //               (zero fill outside the tensor);
 //   warps 3-10  re-lay them into the K-major "4 channels x slot" operand layout of the MMA,
 //               rounding fp32 to TF32 (nearest) and writing zeros for padding;
-//   warp 1      streams the pre-packed, pre-rounded weights of (channel block, tap) by bulk copy;
+//   warp 1      streams the pre-packed, pre-rounded weights by bulk copy;
 //   warp 2      issues, for every tap, tcgen05.mma on the SAME activation tile at a start address
 //               shifted by the tap's slot offset, accumulating in TMEM;
 // then warps 3-10 read the accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
@@ -17,6 +17,8 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.h"
@@ -33,7 +35,8 @@ using namespace tc;
 constexpr int kThreads = 352;              // 11 warps
 constexpr int kXformWarps = 8;
 constexpr int kXformThreads = kXformWarps * 32;
-constexpr int kMaxBStages = 6;
+constexpr int kOwned = 8;                  // slots of an A stage one transform thread may own
+constexpr int kMaxBStages = 12;
 constexpr int kSmemLimit = 232448;
 constexpr int kBarBytes = 512;
 constexpr int kSegBytes = 256;             // >= sizeof(TcConvSegs)
@@ -47,35 +50,58 @@ struct Bars {
 };
 static_assert(sizeof(Bars) <= kBarBytes, "barrier block too large");
 
+#ifdef ONNXB_PROFILE
+__device__ long long g_prof[148 * 16];
+#define PROF_DECL long long pt_ = clock64(), pacc_[5] = {0, 0, 0, 0, 0}
+#define PROF_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
+#define PROF_RESET() do { pt_ = clock64(); } while (0)
+#define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 5; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
+#else
+#define PROF_DECL do {} while (0)
+#define PROF_MARK(k) do {} while (0)
+#define PROF_RESET() do {} while (0)
+#define PROF_FLUSH(base) do {} while (0)
+#endif
+
+// fp32 -> TF32, round to nearest with ties away from zero (what cvt.rna.tf32.f32 computes), done
+// with two integer operations: add half an ulp of the 10-bit mantissa to the magnitude and clear
+// the 13 low bits.  A carry out of the mantissa correctly bumps the exponent; Inf stays Inf.
 __device__ __forceinline__ float round_tf32(float x) {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-    return __uint_as_float(u);
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
+#ifdef ONNXB_CHECK
+__device__ long long g_chk[8];
+#define CHK(cond, code, val) if (!(cond)) { if (atomicCAS((unsigned long long *)&g_chk[0], 0ull, (unsigned long long)(code)) == 0ull) { g_chk[1] = (long long)(val); g_chk[2] = blockIdx.x; g_chk[3] = threadIdx.x; } continue; }
+#else
+#define CHK(cond, code, val)
+#endif
+
 // ------------------------------------------------------------------ weight packing
-// Packed layout: [group][channel tile][channel block][tap][chunk of 4 channels][row BN][4],
-// i.e. for each (channel block, tap) the exact shared-memory image of the K-major operand:
-// 16-byte chunks of 4 consecutive input channels, rows 16 bytes apart.  Values are rounded
-// to TF32 (nearest); rows past the group's channels and channels past Cg are zero.
+// Packed layout: [group][channel tile][channel block][K-step][chunk 0/1][row BN][4], i.e. for each
+// K-step the exact shared-memory image of the K-major B operand: two 16-byte chunks (4 reduction
+// terms each) per output channel, rows 16 bytes apart.  Values are rounded to TF32 (nearest);
+// rows past the group's channels, channels past Cg and unpaired taps are zero.
 __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict__ W, float4 *__restrict__ out) {
     const long long total = g.packed_floats / 4;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
         long long t = i;
         const int row = (int)(t % g.BN); t /= g.BN;
-        const int chunk = (int)(t % (kConvKB / 4)); t /= (kConvKB / 4);
-        const int tap = (int)(t % g.taps); t /= g.taps;
+        const int k = (int)(t % 2); t /= 2;
+        const int step = (int)(t % g.n_steps); t /= g.n_steps;
         const int cb = (int)(t % g.ncb); t /= g.ncb;
         const int ct = (int)(t % g.ctiles); t /= g.ctiles;
         const int grp = (int)t;
         const int mg = ct * g.BN + row;
+        const int tap = g.src_tap[step][k];
         float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (mg < g.Mg) {
+        if (mg < g.Mg && tap >= 0) {
             const int m = grp * g.Mg + mg;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int c = cb * kConvKB + chunk * 4 + e;
+                const int c = cb * g.KB + g.src_c0[step][k] + e;
+                CHK(((size_t)m * g.Cg + (c < g.Cg ? c : 0)) * g.taps + tap < (size_t)g.M * g.Cg * g.taps, 1, ((size_t)m * g.Cg + c) * g.taps + tap)
                 if (c < g.Cg) v[e] = round_tf32(__ldg(W + ((size_t)m * g.Cg + c) * g.taps + tap));
             }
         }
@@ -89,7 +115,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                const float *__restrict__ Wpk, const float *__restrict__ bias, float *__restrict__ Y,
                unsigned int *err) {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler
+    // keeps treating everything derived from it as shared memory (LDS/STS, not generic accesses)
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *a_st = smem;
     uint8_t *raw_st = a_st + 2 * (size_t)g.a_stage_bytes;
     uint8_t *b_st = raw_st + 2 * (size_t)g.raw_stage_bytes;
@@ -129,48 +157,61 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         if (elect_one()) {
             int rs = 0;
             uint32_t rphase = 0;
+            const long long HW = (long long)g.H * g.W;
+            const long long planes_total = (long long)g.N * g.C;
+            const int KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP;
             for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
                 const int ct_all = (int)(t % (g.ctiles * g.group));
                 const int grp = ct_all / g.ctiles;
                 const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
-                for (int cb = 0; cb < g.ncb; ++cb) {
+                // The segment table is the same for every channel block of the tile.  It lives beside
+                // the raw stage that carries the tile's first block and is written only once that stage
+                // has been released, so it cannot change under transform warps still working on an
+                // earlier tile; they read it after this stage has landed.
+                TcConvSegs *segs = nullptr;
+                int nseg = 0;
+                uint32_t tile_bytes = 0;
+                for (int cb = 0; cb < ncb; ++cb) {
                     mbar_wait(&bars->raw_empty[rs], rphase ^ 1, err, 11);
-                    TcConvSegs *segs = reinterpret_cast<TcConvSegs *>(seg_st + rs * kSegBytes);
-                    tc_conv_segments(g, G0, *segs);
+                    if (cb == 0) {
+                        segs = reinterpret_cast<TcConvSegs *>(seg_st + rs * kSegBytes);
+                        tc_conv_segments(g, G0, *segs);
+                        nseg = segs->nseg;
+                        tile_bytes = (uint32_t)segs->total_floats * 4u;
+                    }
                     float *dst = reinterpret_cast<float *>(raw_st + (size_t)rs * g.raw_stage_bytes);
-                    const int c0 = grp * g.Cg + cb * kConvKB;
+                    const int c0 = grp * g.Cg + cb * KB;
                     if (g.raw_mode == 0) {
-                        mbar_arrive_expect_tx(&bars->raw_full[rs], (uint32_t)segs->total_floats * 4u);
-                        for (int i = 0; i < segs->nseg; ++i) {
+                        mbar_arrive_expect_tx(&bars->raw_full[rs], tile_bytes);
+                        for (int i = 0; i < nseg; ++i) {
                             const int plane0 = (segs->n_first + i) * g.C + c0;
-                            for (int j = 0; j < segs->nbox[i]; ++j)
-                                tma_load_2d(dst + segs->base[i] + j * (kConvKB * g.BOXP), &tmX, &bars->raw_full[rs],
-                                            segs->f0[i] + j * g.BOXP, plane0);
+                            const int nbox = segs->nbox[i], f0 = segs->f0[i];
+                            float *d = dst + segs->base[i];
+                            for (int j = 0; j < nbox; ++j)
+                                tma_load_2d(d + j * box_floats, &tmX, &bars->raw_full[rs], f0 + j * g.BOXP, plane0);
                         }
                     } else {
                         // whole-image slabs [channel][H*W]; clip at the end of X
-                        const long long HW = (long long)g.H * g.W;
-                        const long long planes_total = (long long)g.N * g.C;
-                        uint32_t bytes[kConvMaxSeg];
                         uint32_t total = 0;
-                        for (int i = 0; i < segs->nseg; ++i) {
-                            bytes[i] = 0;
-                            if (segs->nbox[i]) {
-                                const long long plane0 = (long long)(segs->n_first + i) * g.C + c0;
-                                long long nch = planes_total - plane0;
-                                if (nch > kConvKB) nch = kConvKB;
-                                bytes[i] = nch > 0 ? (uint32_t)(nch * HW * 4) : 0u;
-                                total += bytes[i];
-                            }
+                        for (int i = 0; i < nseg; ++i) {
+                            if (!segs->nbox[i]) continue;
+                            long long nch = planes_total - ((long long)(segs->n_first + i) * g.C + c0);
+                            if (nch > KB) nch = KB;
+                            if (nch > 0) total += (uint32_t)(nch * HW * 4);
                         }
                         mbar_arrive_expect_tx(&bars->raw_full[rs], total);
-                        for (int i = 0; i < segs->nseg; ++i)
-                            if (bytes[i])
-                                bulk_load_1d(dst + segs->base[i],
-                                             X + ((long long)(segs->n_first + i) * g.C + c0) * HW, bytes[i],
+                        for (int i = 0; i < nseg; ++i) {
+                            if (!segs->nbox[i]) continue;
+                            const long long plane0 = (long long)(segs->n_first + i) * g.C + c0;
+                            long long nch = planes_total - plane0;
+                            if (nch > KB) nch = KB;
+                            if (nch > 0)
+                                bulk_load_1d(dst + segs->base[i], X + plane0 * HW, (uint32_t)(nch * HW * 4),
                                              &bars->raw_full[rs]);
+                        }
                     }
-                    if (++rs == 2) { rs = 0; rphase ^= 1; }
+                    rs ^= 1;
+                    if (rs == 0) rphase ^= 1;
                 }
             }
         }
@@ -179,60 +220,76 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         if (elect_one()) {
             int bs = 0;
             uint32_t bphase = 0;
-            const long long per_ct = (long long)g.ncb * g.taps * g.BN * kConvKB;   // floats per channel tile
+            const long long per_ct = (long long)g.ncb * g.n_steps * g.b_step_bytes;   // bytes per channel tile
+            const int nb = g.nb_stages, ncb = g.ncb, b_steps = g.b_steps, spb = g.spb, n_steps = g.n_steps;
+            const uint32_t stage_bytes = (uint32_t)g.b_stage_bytes, step_bytes = (uint32_t)g.b_step_bytes;
             for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
                 const int ct_all = (int)(t % (g.ctiles * g.group));
-                const float *src = Wpk + ct_all * per_ct;
-                for (int step = 0; step < g.ncb * g.taps; ++step) {
-                    mbar_wait(&bars->b_empty[bs], bphase ^ 1, err, 12);
-                    mbar_arrive_expect_tx(&bars->b_full[bs], (uint32_t)g.b_stage_bytes);
-                    bulk_load_1d(b_st + (size_t)bs * g.b_stage_bytes, src + (long long)step * g.BN * kConvKB,
-                                 (uint32_t)g.b_stage_bytes, &bars->b_full[bs]);
-                    if (++bs == g.nb_stages) { bs = 0; bphase ^= 1; }
+                const uint8_t *src = reinterpret_cast<const uint8_t *>(Wpk) + ct_all * per_ct;
+                for (int cb = 0; cb < ncb; ++cb) {
+                    for (int bstep = 0; bstep < b_steps; ++bstep) {
+                        const uint32_t bytes = (uint32_t)min(spb, n_steps - bstep * spb) * step_bytes;
+                        mbar_wait(&bars->b_empty[bs], bphase ^ 1, err, 12);
+                        mbar_arrive_expect_tx(&bars->b_full[bs], bytes);
+                        bulk_load_1d(b_st + (size_t)bs * stage_bytes, src, bytes, &bars->b_full[bs]);
+                        src += bytes;
+                        if (++bs == nb) { bs = 0; bphase ^= 1; }
+                    }
                 }
             }
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------ MMA issuer
+        // One thread issues every MMA.  Operands are no-swizzle K-major: rows 16 bytes apart, 8-row
+        // groups 128 bytes apart (SBO), the two 16-byte K chunks of one instruction LBO apart.  For
+        // A the per-step table holds offset and LBO (a chunk pitch, or the distance between two taps);
+        // all descriptor words are precomputed, a step costs a table read and a few adds.
         if (elect_one()) {
+            const uint32_t desc_hi = (128u >> 4) | (1u << 14);                 // SBO = 128, descriptor version 1
+            const uint32_t a_base16 = (smem_u32(a_st) >> 4) & 0x3FFFu;
+            const uint32_t b_lo0 = ((smem_u32(b_st) >> 4) & 0x3FFFu) | (((uint32_t)g.BN * 16u >> 4) << 16);
+            const uint32_t a_stage16 = (uint32_t)g.a_stage_bytes >> 4, b_stage16 = (uint32_t)g.b_stage_bytes >> 4;
+            const uint32_t b_step16 = (uint32_t)g.b_step_bytes >> 4;
+            const uint32_t idesc = g.idesc;
+            const int n_steps = g.n_steps, ncb = g.ncb, nb = g.nb_stages, spb = g.spb, b_steps = g.b_steps;
+            const bool two = g.MT == 2;
             int as = 0, bs = 0;
             uint32_t aphase = 0, bphase = 0, accphase = 0;
+            PROF_DECL;
             for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
                 mbar_wait(&bars->acc_empty, accphase ^ 1, err, 13);
                 tc_fence_after_sync();
+                PROF_MARK(0);
                 uint32_t accumulate = 0;
-                for (int cb = 0; cb < g.ncb; ++cb) {
+                for (int cb = 0; cb < ncb; ++cb) {
                     mbar_wait(&bars->a_full[as], aphase, err, 14);
-                    const uint32_t a_base = smem_u32(a_st + (size_t)as * g.a_stage_bytes);
-                    for (int tap = 0; tap < g.taps; ++tap) {
+                    PROF_MARK(1);
+                    const uint32_t a_lo = a_base16 + (uint32_t)as * a_stage16;
+                    for (int bstep = 0; bstep < b_steps; ++bstep) {
                         mbar_wait(&bars->b_full[bs], bphase, err, 15);
                         tc_fence_after_sync();
-                        const uint32_t b_base = smem_u32(b_st + (size_t)bs * g.b_stage_bytes);
-                        const uint32_t a_tap = a_base + (uint32_t)g.tap_plane[tap] * g.plane_pitch +
-                                               (uint32_t)g.tap_shift[tap] * 16u;
-#pragma unroll
-                        for (int j = 0; j < kConvKB / 8; ++j) {
-                            // no-swizzle K-major operands: rows 16 bytes apart (8-row groups 128 bytes
-                            // apart), the two 16-byte K chunks of one instruction one chunk pitch apart
-                            const uint64_t bd = make_smem_desc(b_base + (uint32_t)(2 * j) * g.BN * 16u,
-                                                               (uint32_t)g.BN * 16u, 128, kSwizzleNone);
-                            for (int mt = 0; mt < g.MT; ++mt) {
-                                const uint64_t ad =
-                                    make_smem_desc(a_tap + (uint32_t)(2 * j) * g.chunk_pitch + (uint32_t)mt * 2048u,
-                                                   (uint32_t)g.chunk_pitch, 128, kSwizzleNone);
-                                mma_tf32(tmem_base + (uint32_t)mt * 256u, ad, bd, g.idesc, accumulate);
-                            }
+                        PROF_MARK(2);
+                        const int s0 = bstep * spb, s1 = min(n_steps, s0 + spb);
+                        uint32_t bl = b_lo0 + (uint32_t)bs * b_stage16;
+                        for (int s = s0; s < s1; ++s, bl += b_step16) {
+                            const uint32_t al = a_lo + g.step_a[s];
+                            mma_tf32_lohi(tmem_base, al, desc_hi, bl, desc_hi, idesc, accumulate);
+                            if (two) mma_tf32_lohi(tmem_base + 256u, al + 128u, desc_hi, bl, desc_hi, idesc, accumulate);
                             accumulate = 1;
                         }
                         mma_commit(&bars->b_empty[bs]);
-                        if (++bs == g.nb_stages) { bs = 0; bphase ^= 1; }
+                        if (++bs == nb) { bs = 0; bphase ^= 1; }
+                        PROF_MARK(3);
                     }
                     mma_commit(&bars->a_empty[as]);
-                    if (++as == 2) { as = 0; aphase ^= 1; }
+                    as ^= 1;
+                    if (as == 0) aphase ^= 1;
                 }
                 mma_commit(&bars->acc_full);
                 accphase ^= 1;
+                PROF_MARK(4);
             }
+            PROF_FLUSH(0);
         }
     } else {
         // ------------------------------------------------------------ transform + epilogue warps
@@ -242,20 +299,24 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         const int hf = xw >> 2;
         const int cp = g.raw_mode == 1 ? g.H * g.W : g.BOXP;    // channel pitch inside the raw stage
         const int per_stage_slots = g.planes * g.SLOTS;
+        const int nchunks = g.nchunks, KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP;
+        const uint32_t chunk_pitch = (uint32_t)g.chunk_pitch;
         const long long PQ = (long long)g.P * g.Q;
         int rs = 0, as = 0;
         uint32_t rphase = 0, aphase = 0, accphase = 0;
+        PROF_DECL;
         for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
             const int ct_all = (int)(t % (g.ctiles * g.group));
             const int grp = ct_all / g.ctiles, ct = ct_all % g.ctiles;
             const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
-            int off[4];                            // raw float offset of channel 0 for up to 4 owned slots
-            for (int cb = 0; cb < g.ncb; ++cb) {
+            int off[kOwned];                       // raw float offset of channel 0 for the slots this thread owns
+            for (int cb = 0; cb < ncb; ++cb) {
                 mbar_wait(&bars->raw_full[rs], rphase, err, 16);
+                PROF_MARK(0);
                 if (cb == 0) {
                     const TcConvSegs *segs = reinterpret_cast<const TcConvSegs *>(seg_st + rs * kSegBytes);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                    for (int i = 0; i < kOwned; ++i) {
                         off[i] = -1;
                         const int idx = xt + i * kXformThreads;
                         if (idx < per_stage_slots) {
@@ -268,28 +329,29 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                                 const int h = hq * g.sh + g.pa[pl] - g.pt;
                                 const int w = wq * g.sw + g.pb[pl] - g.pl;
                                 const int sg = n - segs->n_first;
-                                if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && sg < segs->nseg) {
+                                if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
                                     const int f = h * g.W + w - segs->f0[sg];
                                     if (g.raw_mode == 1) off[i] = segs->base[sg] + f;
                                     else {
                                         const int bx = f / g.BOXP;
-                                        off[i] = segs->base[sg] + bx * (kConvKB * g.BOXP) + (f - bx * g.BOXP);
+                                        off[i] = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
                                     }
                                 }
                             }
                         }
                     }
+                    PROF_MARK(2);
                 }
                 mbar_wait(&bars->a_empty[as], aphase ^ 1, err, 17);
+                PROF_MARK(1);
                 const float *raw = reinterpret_cast<const float *>(raw_st + (size_t)rs * g.raw_stage_bytes);
                 uint8_t *adst = a_st + (size_t)as * g.a_stage_bytes;
-                const int c_left = g.Cg - cb * kConvKB;    // channels of this block that exist
+                const int c_left = g.Cg - cb * KB;     // channels of this block that exist
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < kOwned; ++i) {
                     const int idx = xt + i * kXformThreads;
                     if (idx < per_stage_slots) {
-#pragma unroll
-                        for (int ch = 0; ch < kConvKB / 4; ++ch) {
+                        for (int ch = 0; ch < nchunks; ++ch) {
                             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                             if (off[i] >= 0) {
                                 const float *r = raw + off[i] + (ch * 4) * cp;
@@ -299,57 +361,71 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                                 if (left > 2) v.z = round_tf32(r[2 * cp]);
                                 if (left > 3) v.w = round_tf32(r[3 * cp]);
                             }
-                            *reinterpret_cast<float4 *>(adst + (size_t)ch * g.chunk_pitch + (size_t)idx * 16) = v;
+                            *reinterpret_cast<float4 *>(adst + (size_t)ch * chunk_pitch + (size_t)idx * 16) = v;
                         }
                     }
                 }
+                PROF_MARK(2);
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(&bars->a_full[as]);
                     mbar_arrive(&bars->raw_empty[rs]);
                 }
-                if (++rs == 2) { rs = 0; rphase ^= 1; }
-                if (++as == 2) { as = 0; aphase ^= 1; }
+                PROF_MARK(3);
+                rs ^= 1;
+                if (rs == 0) rphase ^= 1;
+                as ^= 1;
+                if (as == 0) aphase ^= 1;
             }
 
             // ---- epilogue of this tile
             mbar_wait(&bars->acc_full, accphase, err, 18);
             tc_fence_after_sync();
+            PROF_RESET();
             const int nch = (g.BN + 31) / 32;
             int mt, ch_lo, ch_hi;
             if (g.MT == 2) { mt = hf; ch_lo = 0; ch_hi = nch; }
             else { mt = 0; ch_lo = hf ? (nch + 1) / 2 : 0; ch_hi = hf ? nch : (nch + 1) / 2; }
             const long long G = G0 + mt * 128 + quarter * 32 + lane;
             bool valid = G < g.total_slots;
-            long long ybase = 0;
+            float *yrow = Y;
             if (valid) {
                 const int n = (int)(G / g.L);
                 const int u = (int)(G - (long long)n * g.L);
                 const int p = u / g.Ws, q = u - p * g.Ws;
                 valid = p < g.P && q < g.Q;
-                ybase = ((long long)n * g.M * g.P + p) * g.Q + q;
+                yrow = Y + ((long long)n * g.M * g.P + p) * g.Q + q;
             }
+            const int m_lim = min(g.Mg, (ct + 1) * g.BN);          // channels of this tile that exist
             for (int chunk = ch_lo; chunk < ch_hi; ++chunk) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * 256 + chunk * 32), v);
+                const int mg0 = ct * g.BN + chunk * 32;            // first channel (within the group) of the chunk
+                // lane j fetches the bias of column j once; columns then take it by shuffle
+                const float bl = (bias && mg0 + lane < m_lim) ? __ldg(bias + grp * g.Mg + mg0 + lane) : 0.f;
+                float *yp = yrow + (long long)(grp * g.Mg + mg0) * PQ;
                 tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const int mg = ct * g.BN + chunk * 32 + j;     // channel within the group (warp-uniform)
-                    if (mg < g.Mg && chunk * 32 + j < g.BN) {
-                        const int m = grp * g.Mg + mg;
-                        float x = __uint_as_float(v[j]) + (bias ? __ldg(bias + m) : 0.f);
-                        if (g.relu) x = x > 0.f ? x : 0.f;
-                        if (valid) Y[ybase + (long long)m * PQ] = x;
+                    float x = __uint_as_float(v[j]) + __shfl_sync(0xffffffffu, bl, j);
+                    if (g.relu) x = x > 0.f ? x : 0.f;
+#ifdef ONNXB_CHECK
+                    if (valid && mg0 + j < m_lim) {
+                        const long long yi = (yp + (long long)j * PQ) - Y;
+                        CHK(yi >= 0 && yi < (long long)g.N * g.M * PQ, 2, yi)
                     }
+#endif
+                    if (valid && mg0 + j < m_lim) yp[(long long)j * PQ] = x;
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->acc_empty);
             accphase ^= 1;
+            PROF_MARK(4);
         }
+        if (xt == 0) PROF_FLUSH(5);
     }
 
     tc_fence_before_sync();
@@ -425,22 +501,71 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     for (int i = 0; i < ah.npar; ++i)
         for (int j = 0; j < aw.npar; ++j) { g.pa[g.planes] = ah.par[i]; g.pb[g.planes] = aw.par[j]; ++g.planes; }
     g.a_min = ah.par[0]; g.a_max = ah.par[ah.npar - 1];
+    const long long maxshift = (long long)ah.Amax * g.Ws + aw.Amax;
+    g.MT = MT; g.BN = BN;
+    g.ctiles = (c.Mg + BN - 1) / BN;
+    const long long slots = (long long)MT * 128 + maxshift;
+    if (slots * g.planes > kOwned * kXformThreads) return false;
+    g.SLOTS = (int)slots;
+    if ((g.SLOTS + L - 2) / L + 1 > kConvMaxSeg) return false;
+    g.plane_pitch = g.SLOTS * 16;
+    g.chunk_pitch = g.planes * g.plane_pitch;
+    if (g.chunk_pitch >= (1 << 18)) return false;
+
+    // per-tap plane and slot shift, in 16-byte units inside an A stage
+    int tap_plane[kConvMaxTaps], tap_off16[kConvMaxTaps];
     for (int r = 0; r < c.kH; ++r)
         for (int s = 0; s < c.kW; ++s) {
             const int a = (r * c.dh) % c.sh, b = (s * c.dw) % c.sw;
             int pl = 0;
             while (g.pa[pl] != a || g.pb[pl] != b) ++pl;
-            g.tap_plane[r * c.kW + s] = pl;
-            g.tap_shift[r * c.kW + s] = ((r * c.dh) / c.sh) * g.Ws + (s * c.dw) / c.sw;
+            const int shift = ((r * c.dh) / c.sh) * g.Ws + (s * c.dw) / c.sw;
+            tap_plane[r * c.kW + s] = pl;
+            tap_off16[r * c.kW + s] = (pl * g.plane_pitch + shift * 16) >> 4;
         }
-    const long long maxshift = (long long)ah.Amax * g.Ws + aw.Amax;
-    g.MT = MT; g.BN = BN;
-    g.ctiles = (c.Mg + BN - 1) / BN;
-    const long long slots = (long long)MT * 128 + maxshift;
-    if (slots * g.planes > 4 * kXformThreads) return false;      // each transform thread owns at most 4 slots
-    g.SLOTS = (int)slots;
-    if ((g.SLOTS + L - 2) / L + 1 > kConvMaxSeg) return false;
-    g.ncb = (c.Cg + kConvKB - 1) / kConvKB;
+
+    // K-steps of one channel block
+    if (c.Cg >= 16) {
+        g.KB = 16;
+        g.n_steps = 2 * g.taps;
+        const uint32_t lbo16 = (uint32_t)g.chunk_pitch >> 4;
+        if (lbo16 >= (1u << 14)) return false;
+        for (int tp = 0; tp < g.taps; ++tp)
+            for (int j = 0; j < 2; ++j) {
+                const int s = 2 * tp + j;
+                g.step_a[s] = ((uint32_t)tap_off16[tp] + (uint32_t)j * 2u * lbo16) | (lbo16 << 16);
+                g.src_tap[s][0] = g.src_tap[s][1] = (short)tp;
+                g.src_c0[s][0] = (short)(j * 8);
+                g.src_c0[s][1] = (short)(j * 8 + 4);
+            }
+    } else {
+        // tap pairs: within each plane, taps in order of their offset, two per step
+        g.KB = 4;
+        g.n_steps = 0;
+        for (int pl = 0; pl < g.planes; ++pl) {
+            int list[kConvMaxTaps], n = 0;
+            for (int tp = 0; tp < g.taps; ++tp)
+                if (tap_plane[tp] == pl) list[n++] = tp;
+            std::sort(list, list + n, [&](int x, int y) { return tap_off16[x] < tap_off16[y]; });
+            for (int i = 0; i < n; i += 2) {
+                const int t0 = list[i], t1 = i + 1 < n ? list[i + 1] : -1;
+                const uint32_t lbo16 = t1 >= 0 ? (uint32_t)(tap_off16[t1] - tap_off16[t0]) : 0u;
+                if (lbo16 >= (1u << 14)) return false;
+                const int s = g.n_steps++;
+                g.step_a[s] = (uint32_t)tap_off16[t0] | (lbo16 << 16);
+                g.src_tap[s][0] = (short)t0;
+                g.src_tap[s][1] = (short)t1;
+                g.src_c0[s][0] = g.src_c0[s][1] = 0;
+            }
+        }
+    }
+    for (int s = g.n_steps; s < kConvMaxSteps; ++s) {
+        g.step_a[s] = 0;
+        g.src_tap[s][0] = g.src_tap[s][1] = -1;
+        g.src_c0[s][0] = g.src_c0[s][1] = 0;
+    }
+    g.nchunks = g.KB / 4;
+    g.ncb = (c.Cg + g.KB - 1) / g.KB;
     const long long ptiles = (g.total_slots + MT * 128 - 1) / (MT * 128);
     if (ptiles > 0x7fffffffLL) return false;
     g.pix_tiles = (int)ptiles;
@@ -449,46 +574,47 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     const long long HW = (long long)c.H * c.W;
     if (HW % 4 == 0) {
         g.raw_mode = 0;
-    } else if (c.Cg % 4 == 0 && c.C % 4 == 0 && HW * kConvKB * 4 <= 32768) {
+    } else if (c.Cg % 4 == 0 && c.C % 4 == 0 && HW * g.KB * 4 <= 32768) {
         g.raw_mode = 1;
     } else {
         return false;
     }
-    g.plane_pitch = g.SLOTS * 16;
-    g.chunk_pitch = g.planes * g.plane_pitch;
-    if (g.chunk_pitch >= (1 << 18)) return false;
-    g.a_stage_bytes = (kConvKB / 4) * g.chunk_pitch;
+    g.a_stage_bytes = g.nchunks * g.chunk_pitch;
     g.a_stage_bytes = (g.a_stage_bytes + 127) / 128 * 128;
-    g.b_stage_bytes = BN * kConvKB * 4;
+    g.b_step_bytes = BN * 32;
+    g.spb = std::max(1, std::min(g.n_steps, 32768 / g.b_step_bytes));   // several K-steps per weight stage
     g.idesc = tc::make_idesc_tf32(128, BN, 0, 0);
-    g.packed_floats = (long long)c.group * g.ctiles * g.ncb * g.taps * BN * kConvKB;
+    g.packed_floats = (long long)c.group * g.ctiles * g.ncb * g.n_steps * BN * 8;
     // raw stage size: widest flat pixel range any tile needs, found by walking the tiles
     g.BOXP = 256;
+    const long long walk = std::min<long long>(ptiles, L + 2);
     if (g.raw_mode == 0) {
         int widest = 4;
-        const long long walk = std::min<long long>(ptiles, L + 2);
         for (long long i = 0; i <= walk; ++i) {
             const long long pt = i < walk ? i : ptiles - 1;
             const long long G0 = pt * MT * 128;
-            long long Gend = std::min<long long>(G0 + g.SLOTS, g.total_slots);
+            const long long Gend = std::min<long long>(G0 + g.SLOTS, g.total_slots);
             const int n_first = (int)(G0 / L), n_last = (int)((Gend - 1) / L);
             for (int n = n_first; n <= n_last; ++n) {
                 const long long lo = std::max<long long>(G0, (long long)n * L), hi = std::min<long long>(Gend, (long long)(n + 1) * L);
                 const int hq_lo = (int)((lo - (long long)n * L) / g.Ws), hq_hi = (int)((hi - 1 - (long long)n * L) / g.Ws);
-                int h_min = std::max(0, hq_lo * c.sh + g.a_min - c.pt);
-                int h_max = std::min(c.H - 1, hq_hi * c.sh + g.a_max - c.pt);
+                const int h_min = std::max(0, hq_lo * c.sh + g.a_min - c.pt);
+                const int h_max = std::min(c.H - 1, hq_hi * c.sh + g.a_max - c.pt);
                 if (h_min > h_max) continue;
                 const int f0 = (h_min * c.W) & ~3;
                 widest = std::max(widest, (h_max + 1) * c.W - f0);
             }
         }
+        // boxes of <= 256 pixels, split evenly; every box must start on a 128-byte boundary of
+        // shared memory (TMA destination alignment), i.e. KB * BOXP * 4 bytes is a multiple of 128
+        const int align = std::max(4, 32 / g.KB);
         widest = (widest + 3) / 4 * 4;
-        g.BOXP = std::min(256, widest);
+        const int nbox = (widest + 255) / 256;
+        g.BOXP = std::min(256, ((widest + nbox - 1) / nbox + align - 1) / align * align);
     }
     {
         int worst = 0;
         TcConvSegs segs;
-        const long long walk = std::min<long long>(ptiles, L + 2);
         for (long long i = 0; i <= walk; ++i) {
             const long long pt = i < walk ? i : ptiles - 1;
             tc_conv_segments(g, pt * MT * 128, segs);
@@ -499,6 +625,9 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     }
     const long long fixed = 1024 + 2LL * g.a_stage_bytes + 2LL * g.raw_stage_bytes + 2 * kSegBytes + kBarBytes;
     const long long room = kSmemLimit - fixed;
+    while (room < 3LL * g.spb * g.b_step_bytes && g.spb > 1) g.spb = (g.spb + 1) / 2;   // keep three stages in flight
+    g.b_steps = (g.n_steps + g.spb - 1) / g.spb;
+    g.b_stage_bytes = g.spb * g.b_step_bytes;
     if (room < 2LL * g.b_stage_bytes) return false;
     g.nb_stages = (int)std::min<long long>(kMaxBStages, room / g.b_stage_bytes);
     return true;
@@ -506,12 +635,16 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
 
 }  // namespace
 
-bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan) {
-    if (c.Cg < 16) return false;                  // thin contraction: SIMT family
+bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
+    const long long taps = (long long)c.kH * c.kW;
+    if (c.Cg < 16) {
+        // tap-pair mode needs at least two taps, and is kept for problems big enough to matter:
+        // tiny thin contractions (an MNIST-size first layer) stay on the exact fp32 SIMT kernel
+        const double flops = 2.0 * c.N * c.M * c.P * c.Q * c.Cg * (double)taps;
+        if (taps < 2 || c.Cg * taps < 32 || (flops < 5e7 && !forced)) return false;
+    }
     const int sms = 148;
     const int bn0 = pick_conv_bn(c.Mg);
-    // Candidate tiles, largest first: 256 or 128 pixels x up to 256 channels.  The cost model is
-    // waves x (MMA time of one tile, with a floor where narrow tiles become shared-memory bound).
     int cand[5][2];
     int ncand = 0;
     cand[ncand][0] = 2; cand[ncand++][1] = bn0;
@@ -526,8 +659,18 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan) {
     for (int i = 0; i < ncand; ++i) {
         TcConvPlan p;
         if (!fill_plan(c, cand[i][0], cand[i][1], p)) continue;
+        // Cost in SM cycles.  Per channel block the slowest of: the transform warps (about 200 + 420
+        // cycles per 256 slots and chunk quartet), the tensor pipe (BN/2 cycles per instruction, or the
+        // shared-memory time of its operands when that is longer) and the weight stream out of L2
+        // (about 3600 bytes per cycle over all SMs, at most 64 per SM).
         const long long waves = (p.total_tiles + sms - 1) / sms;
-        const double cost = (double)waves * p.MT * std::max(p.BN, 96);
+        const double active = (double)std::min<long long>(p.total_tiles, sms);
+        const double t_x = (200.0 + 420.0 * ((p.planes * p.SLOTS + 255) / 256)) * p.nchunks / 4.0;
+        const double t_inst = std::max(p.BN / 2.0, 40.0 + p.BN / 4.0) * (p.BN <= 128 ? 1.25 : 1.0);
+        const double t_mma = (double)p.n_steps * p.MT * t_inst;
+        const double t_w = (double)p.n_steps * p.b_step_bytes / std::min(64.0, 3600.0 / active);
+        const double per_cb = std::max(t_x, std::max(t_mma, t_w));
+        const double cost = (double)waves * (p.ncb * per_cb + 3000.0 + 8.0 * p.MT * p.BN);
         if (!have || cost < best_cost * 0.999) {
             have = true;
             best_cost = cost;
@@ -536,6 +679,21 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan) {
     }
     return have;
 }
+
+#ifdef ONNXB_CHECK
+extern "C" int onnxb_dbg_check(long long *out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_chk, sizeof(long long) * 8);
+    return 0;
+}
+#endif
+#ifdef ONNXB_PROFILE
+extern "C" int onnxb_dbg_profile(long long *out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 148 * 16);
+    return 0;
+}
+#endif
 
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan) { return (size_t)plan.packed_floats * 4; }
 
@@ -560,7 +718,7 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     if (plan.raw_mode == 0) {
         const uint64_t dims[2] = {(uint64_t)plan.H * plan.W, (uint64_t)plan.N * plan.C};
         const uint64_t str[1] = {(uint64_t)plan.H * plan.W * 4};
-        const uint32_t box[2] = {(uint32_t)plan.BOXP, (uint32_t)kConvKB};
+        const uint32_t box[2] = {(uint32_t)plan.BOXP, (uint32_t)plan.KB};
         if (!make_tmap(&tmX, X, 2, dims, str, box, kTmapSwizzleNone)) return (int)cudaErrorInvalidValue;
     } else {
         memset(&tmX, 0, sizeof tmX);
@@ -571,6 +729,12 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     if (e != cudaSuccess) return (int)e;
     const int sms = num_sms();
     const int grid = (int)std::min<long long>(plan.total_tiles, sms);
+#ifdef ONNXB_PROFILE
+    fprintf(stderr, "[plan] MT %d BN %d ctiles %d SLOTS %d planes %d Hs %d Ws %d L %d KB %d ncb %d steps %d spb %d tiles %lld grid %d raw_mode %d BOXP %d a_stage %d raw_stage %d b_stage %d nb %d smem %zu\n",
+            plan.MT, plan.BN, plan.ctiles, plan.SLOTS, plan.planes, plan.Hs, plan.Ws, plan.L, plan.KB, plan.ncb,
+            plan.n_steps, plan.spb, plan.total_tiles, grid, plan.raw_mode, plan.BOXP, plan.a_stage_bytes,
+            plan.raw_stage_bytes, plan.b_stage_bytes, plan.nb_stages, smem);
+#endif
     tc_conv_kernel<<<grid, kThreads, smem, st>>>(tmX, plan, X, reinterpret_cast<const float *>(workspace), B, Y, err);
     count_launch();
     return (int)cudaGetLastError();

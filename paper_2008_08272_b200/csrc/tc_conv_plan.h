@@ -23,8 +23,8 @@ namespace onnxb {
 
 constexpr int kConvMaxPlanes = 4;
 constexpr int kConvMaxTaps = 64;
+constexpr int kConvMaxSteps = 128;     // MMA K-steps (8 reduction terms each) per channel block
 constexpr int kConvMaxSeg = 8;
-constexpr int kConvKB = 16;            // input channels per pipeline step (four 16-byte chunks)
 
 struct TcConvPlan {
     // problem
@@ -35,19 +35,27 @@ struct TcConvPlan {
     int planes, pa[kConvMaxPlanes], pb[kConvMaxPlanes];
     int a_min, a_max;                // smallest / largest used row parity
     int taps;
-    int tap_plane[kConvMaxTaps], tap_shift[kConvMaxTaps];
+    // Reduction blocking.  A channel block holds KB input channels as KB/4 chunks of 4 (one 16-byte
+    // operand row per slot and chunk).  One MMA K-step consumes two chunks:
+    //   KB = 16 ("channel pairs"): chunks 2j, 2j+1 of the same tap, two steps per tap;
+    //   KB = 4  ("tap pairs", for C/group < 16): the single chunk read at two taps of the same plane.
+    int KB, nchunks, n_steps;
+    uint32_t step_a[kConvMaxSteps];      // A descriptor low word relative to the stage: offset/16 | (LBO/16) << 16
+    short src_tap[kConvMaxSteps][2];     // which filter tap feeds chunk 0 / 1 of the step's weights (-1: zeros)
+    short src_c0[kConvMaxSteps][2];      // and from which channel offset inside the block
     // tiling
     int MT;                          // 128-row accumulator tiles per CTA tile (1 or 2)
     int BN, ctiles;                  // output channels per tile, tiles per group
     int SLOTS;                       // slots per plane held in one A stage = MT*128 + largest tap shift
-    int ncb;                         // channel blocks = ceil(Cg / kConvKB)
+    int ncb;                         // channel blocks = ceil(Cg / KB)
     int pix_tiles;                   // ceil(total_slots / (MT*128))
     long long total_tiles;
     // raw staging
-    int raw_mode;                    // 0: tensor-map boxes [kConvKB][BOXP] over X seen as (H*W, N*C); 1: whole-image slabs
+    int raw_mode;                    // 0: tensor-map boxes [KB][BOXP] over X seen as (H*W, N*C); 1: whole-image slabs
     int BOXP;
     // shared memory carve-up (bytes)
     int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages;
+    int spb, b_step_bytes, b_steps;  // K-steps per weight stage, bytes of one step's weights, weight stages per block
     int chunk_pitch, plane_pitch;    // bytes between 4-channel chunks / parity planes inside an A stage
     uint32_t idesc;
     long long packed_floats;         // size of the packed weight buffer
@@ -87,13 +95,13 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
         } else if (g.raw_mode == 1) {
             t.f0[i] = 0;
             t.nbox[i] = 1;
-            base += kConvKB * g.H * g.W;
+            base += g.KB * g.H * g.W;
         } else {
             const int f0 = (h_min * g.W) & ~3;
             const int len = (h_max + 1) * g.W - f0;
             t.f0[i] = f0;
             t.nbox[i] = (len + g.BOXP - 1) / g.BOXP;
-            base += t.nbox[i] * g.BOXP * kConvKB;
+            base += t.nbox[i] * g.BOXP * g.KB;
         }
     }
     t.total_floats = base;

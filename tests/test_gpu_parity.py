@@ -117,6 +117,40 @@ def test_conv_multi_tile(binding, c, relu):
     assert ratio <= 1.0, ratio
 
 
+# the implicit-GEMM tensor-core kernel forced onto shapes the dispatcher would give to the SIMT
+# family: thin contractions (tap-pair mode, C/group < 16), strides, dilations, groups, ragged sizes
+FORCED_IMPLICIT = [
+    dict(x=(2, 3, 64, 64), w=(32, 3, 7, 7), pads=(3, 3, 3, 3), strides=(2, 2)),
+    dict(x=(2, 8, 32, 32), w=(24, 8, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(2, 4, 32, 32), w=(16, 4, 5, 5), pads=(2, 2, 2, 2)),
+    dict(x=(2, 6, 36, 36), w=(20, 6, 3, 3), pads=(1, 1, 1, 1), strides=(2, 2)),
+    dict(x=(2, 12, 32, 32), w=(20, 12, 3, 3), pads=(2, 2, 2, 2), dilations=(2, 2)),
+    dict(x=(3, 2, 28, 28), w=(8, 2, 5, 5), pads=(2, 2, 2, 2)),
+    dict(x=(2, 16, 24, 28), w=(40, 16, 3, 3), pads=(1, 0, 2, 1), strides=(2, 1)),
+    dict(x=(2, 32, 20, 20), w=(48, 8, 3, 3), pads=(1, 1, 1, 1), group=4),
+    dict(x=(5, 64, 7, 7), w=(70, 64, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(70, 4, 16, 16), w=(16, 4, 3, 3), pads=(1, 1, 1, 1)),
+]
+
+
+@pytest.mark.parametrize("c", FORCED_IMPLICIT, ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+def test_conv_forced_implicit_gemm(binding, c):
+    rng = np.random.default_rng(4242)
+    X = rng.standard_normal(c["x"]).astype(np.float32)
+    W = rng.standard_normal(c["w"]).astype(np.float32)
+    B = rng.standard_normal((c["w"][0],)).astype(np.float32)
+    kw = dict(pads=c.get("pads", (0, 0, 0, 0)), strides=c.get("strides", (1, 1)),
+              dilations=c.get("dilations", (1, 1)), group=c.get("group", 1))
+    binding.set_kernel_override("mma_implicit")
+    try:
+        got, fam = run_conv_gpu(binding, torch, X, W, B, relu=True, **kw)
+    finally:
+        binding.set_kernel_override(None)
+    assert fam == "mma_implicit"
+    want, S = oracle.conv2d(X, W, B, relu=True, **kw)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 def test_conv_auto_pad_and_no_bias(binding):
     rng = np.random.default_rng(5)
     X = rng.standard_normal((2, 6, 13, 11)).astype(np.float32)
