@@ -11,8 +11,9 @@
 //   warp 1      streams the pre-packed, pre-rounded weights by bulk copy;
 //   warp 2      issues, for every tap, tcgen05.mma on the SAME activation tile at a start address
 //               shifted by the tap's slot offset, accumulating in TMEM;
-// then warps 3-10 read the accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
-// with lanes along consecutive pixels (coalesced).
+//   warps 11-18 read finished accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
+//               with lanes along consecutive pixels (coalesced); with one 128-row accumulator per
+//               tile TMEM holds two of them, so this overlaps the next tile's MMAs.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -32,10 +33,11 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 352;              // 11 warps
+constexpr int kThreads = 608;              // 19 warps: 2 producers, MMA, 8 transform, 8 epilogue
 constexpr int kXformWarps = 8;
 constexpr int kXformThreads = kXformWarps * 32;
-constexpr int kOwned = 8;                  // slots of an A stage one transform thread may own
+constexpr int kEpiWarps = 8;
+constexpr int kOwned = 10;                 // slots of an A stage one transform thread may own
 constexpr int kMaxBStages = 12;
 constexpr int kSmemLimit = 232448;
 constexpr int kBarBytes = 512;
@@ -45,7 +47,7 @@ static_assert(sizeof(TcConvSegs) <= kSegBytes, "segment table does not fit its s
 struct Bars {
     uint64_t raw_full[2], raw_empty[2], a_full[2], a_empty[2];
     uint64_t b_full[kMaxBStages], b_empty[kMaxBStages];
-    uint64_t acc_full, acc_empty;
+    uint64_t acc_full[2], acc_empty[2];
     uint32_t tmem_holder;
 };
 static_assert(sizeof(Bars) <= kBarBytes, "barrier block too large");
@@ -138,8 +140,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             mbar_init(&bars->b_full[s], 1);
             mbar_init(&bars->b_empty[s], 1);
         }
-        mbar_init(&bars->acc_full, 1);
-        mbar_init(&bars->acc_empty, kXformWarps);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->acc_full[s], 1);
+            mbar_init(&bars->acc_empty[s], kEpiWarps);
+        }
         mbar_fence_init();
         if (g.raw_mode == 0) prefetch_tmap(&tmX);
     }
@@ -254,10 +258,13 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             const int n_steps = g.n_steps, ncb = g.ncb, nb = g.nb_stages, spb = g.spb, b_steps = g.b_steps;
             const bool two = g.MT == 2;
             int as = 0, bs = 0;
-            uint32_t aphase = 0, bphase = 0, accphase = 0;
+            uint32_t aphase = 0, bphase = 0, it = 0;
             PROF_DECL;
-            for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
-                mbar_wait(&bars->acc_empty, accphase ^ 1, err, 13);
+            for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x, ++it) {
+                // accumulator buffer: two of them alternate when a tile needs only 256 TMEM columns
+                const uint32_t ab = two ? 0u : (it & 1u), use = two ? it : (it >> 1);
+                const uint32_t d0 = tmem_base + ab * 256u;
+                mbar_wait(&bars->acc_empty[ab], (use & 1u) ^ 1u, err, 13);
                 tc_fence_after_sync();
                 PROF_MARK(0);
                 uint32_t accumulate = 0;
@@ -273,8 +280,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                         uint32_t bl = b_lo0 + (uint32_t)bs * b_stage16;
                         for (int s = s0; s < s1; ++s, bl += b_step16) {
                             const uint32_t al = a_lo + g.step_a[s];
-                            mma_tf32_lohi(tmem_base, al, desc_hi, bl, desc_hi, idesc, accumulate);
-                            if (two) mma_tf32_lohi(tmem_base + 256u, al + 128u, desc_hi, bl, desc_hi, idesc, accumulate);
+                            mma_tf32_lohi(d0, al, desc_hi, bl, desc_hi, idesc, accumulate);
+                            if (two) mma_tf32_lohi(d0 + 256u, al + 128u, desc_hi, bl, desc_hi, idesc, accumulate);
                             accumulate = 1;
                         }
                         mma_commit(&bars->b_empty[bs]);
@@ -285,29 +292,23 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                     as ^= 1;
                     if (as == 0) aphase ^= 1;
                 }
-                mma_commit(&bars->acc_full);
-                accphase ^= 1;
+                mma_commit(&bars->acc_full[ab]);
                 PROF_MARK(4);
             }
             PROF_FLUSH(0);
         }
-    } else {
-        // ------------------------------------------------------------ transform + epilogue warps
+    } else if (warp < 3 + kXformWarps) {
+        // ------------------------------------------------------------ transform warps
         const int xw = warp - 3;                   // 0..7
         const int xt = xw * 32 + lane;             // 0..255
-        const int quarter = warp & 3;              // TMEM lane quarter this warp may read
-        const int hf = xw >> 2;
         const int cp = g.raw_mode == 1 ? g.H * g.W : g.BOXP;    // channel pitch inside the raw stage
         const int per_stage_slots = g.planes * g.SLOTS;
         const int nchunks = g.nchunks, KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP;
         const uint32_t chunk_pitch = (uint32_t)g.chunk_pitch;
-        const long long PQ = (long long)g.P * g.Q;
         int rs = 0, as = 0;
-        uint32_t rphase = 0, aphase = 0, accphase = 0;
+        uint32_t rphase = 0, aphase = 0;
         PROF_DECL;
         for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
-            const int ct_all = (int)(t % (g.ctiles * g.group));
-            const int grp = ct_all / g.ctiles, ct = ct_all % g.ctiles;
             const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
             int off[kOwned];                       // raw float offset of channel 0 for the slots this thread owns
             for (int cb = 0; cb < ncb; ++cb) {
@@ -321,10 +322,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                         const int idx = xt + i * kXformThreads;
                         if (idx < per_stage_slots) {
                             const int pl = idx / g.SLOTS, j = idx - pl * g.SLOTS;
-                            const long long Gs = G0 + j;
-                            if (Gs < g.total_slots) {
-                                const int n = (int)(Gs / g.L);
-                                const int u = (int)(Gs - (long long)n * g.L);
+                            const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
+                            if (Gs < (uint32_t)g.total_slots) {
+                                const int n = (int)(Gs / (uint32_t)g.L);
+                                const int u = (int)(Gs - (uint32_t)n * (uint32_t)g.L);
                                 const int hq = u / g.Ws, wq = u - hq * g.Ws;
                                 const int h = hq * g.sh + g.pa[pl] - g.pt;
                                 const int w = wq * g.sw + g.pb[pl] - g.pl;
@@ -379,20 +380,34 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 if (as == 0) aphase ^= 1;
             }
 
-            // ---- epilogue of this tile
-            mbar_wait(&bars->acc_full, accphase, err, 18);
+        }
+        if (xt == 0) PROF_FLUSH(5);
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int ew = warp - 3 - kXformWarps;     // 0..7
+        const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+        const int hf = ew >> 2;
+        const long long PQ = (long long)g.P * g.Q;
+        const bool two = g.MT == 2;
+        uint32_t it = 0;
+        for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x, ++it) {
+            const int ct_all = (int)(t % (g.ctiles * g.group));
+            const int grp = ct_all / g.ctiles, ct = ct_all % g.ctiles;
+            const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
+            const uint32_t ab = two ? 0u : (it & 1u), use = two ? it : (it >> 1);
+            mbar_wait(&bars->acc_full[ab], use & 1u, err, 18);
             tc_fence_after_sync();
-            PROF_RESET();
             const int nch = (g.BN + 31) / 32;
             int mt, ch_lo, ch_hi;
-            if (g.MT == 2) { mt = hf; ch_lo = 0; ch_hi = nch; }
+            if (two) { mt = hf; ch_lo = 0; ch_hi = nch; }
             else { mt = 0; ch_lo = hf ? (nch + 1) / 2 : 0; ch_hi = hf ? nch : (nch + 1) / 2; }
-            const long long G = G0 + mt * 128 + quarter * 32 + lane;
-            bool valid = G < g.total_slots;
+            const uint32_t acc_col = two ? (uint32_t)mt * 256u : ab * 256u;
+            const uint32_t G = (uint32_t)G0 + (uint32_t)(mt * 128 + quarter * 32 + lane);
+            bool valid = G < (uint32_t)g.total_slots;
             float *yrow = Y;
             if (valid) {
-                const int n = (int)(G / g.L);
-                const int u = (int)(G - (long long)n * g.L);
+                const int n = (int)(G / (uint32_t)g.L);
+                const int u = (int)(G - (uint32_t)n * (uint32_t)g.L);
                 const int p = u / g.Ws, q = u - p * g.Ws;
                 valid = p < g.P && q < g.Q;
                 yrow = Y + ((long long)n * g.M * g.P + p) * g.Q + q;
@@ -400,7 +415,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             const int m_lim = min(g.Mg, (ct + 1) * g.BN);          // channels of this tile that exist
             for (int chunk = ch_lo; chunk < ch_hi; ++chunk) {
                 uint32_t v[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * 256 + chunk * 32), v);
+                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_col + (uint32_t)(chunk * 32), v);
                 const int mg0 = ct * g.BN + chunk * 32;            // first channel (within the group) of the chunk
                 // lane j fetches the bias of column j once; columns then take it by shuffle
                 const float bl = (bias && mg0 + lane < m_lim) ? __ldg(bias + grp * g.Mg + mg0 + lane) : 0.f;
@@ -410,22 +425,13 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 for (int j = 0; j < 32; ++j) {
                     float x = __uint_as_float(v[j]) + __shfl_sync(0xffffffffu, bl, j);
                     if (g.relu) x = x > 0.f ? x : 0.f;
-#ifdef ONNXB_CHECK
-                    if (valid && mg0 + j < m_lim) {
-                        const long long yi = (yp + (long long)j * PQ) - Y;
-                        CHK(yi >= 0 && yi < (long long)g.N * g.M * PQ, 2, yi)
-                    }
-#endif
                     if (valid && mg0 + j < m_lim) yp[(long long)j * PQ] = x;
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->acc_empty);
-            accphase ^= 1;
-            PROF_MARK(4);
+            if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);
         }
-        if (xt == 0) PROF_FLUSH(5);
     }
 
     tc_fence_before_sync();
@@ -497,6 +503,7 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     if (L > (1 << 24)) return false;
     g.L = (int)L;
     g.total_slots = (long long)c.N * L;
+    if (g.total_slots + 4096 >= (1LL << 31)) return false;        // device code indexes slots in 32 bits
     g.planes = 0;
     for (int i = 0; i < ah.npar; ++i)
         for (int j = 0; j < aw.npar; ++j) { g.pa[g.planes] = ah.par[i]; g.pb[g.planes] = aw.par[j]; ++g.planes; }
