@@ -424,8 +424,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float x = __uint_as_float(v[j]) + __shfl_sync(0xffffffffu, bl, j);
-                    if (g.relu) x = x > 0.f ? x : 0.f;
-                    if (valid && mg0 + j < m_lim) yp[(long long)j * PQ] = x;
+                    if (g.relu) x = fmaxf(x, 0.f);
+                    if (valid && mg0 + j < m_lim) *yp = x;
+                    yp += PQ;
                 }
             }
             tc_fence_before_sync();

@@ -41,6 +41,17 @@ constexpr int kStagingBytes = 4 * 2 * kStoreBufBytes;
 constexpr int kBarrierBytes = 256;
 constexpr int kSmemLimit = 232448;                 // 227 KB opt-in maximum per CTA
 
+#ifdef ONNXB_PROFILE
+__device__ long long g_gprof[148 * 16];
+#define GP_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
+#define GP_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
+#define GP_FLUSH(base, n) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < n; ++k_) g_gprof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
+#else
+#define GP_DECL do {} while (0)
+#define GP_MARK(k) do {} while (0)
+#define GP_FLUSH(base, n) do {} while (0)
+#endif
+
 struct Params {
     int M, N, K, batch;
     int a_mn, b_mn;            // operand is MN-major (else K-major)
@@ -134,13 +145,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
+            GP_DECL;
             for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
                 mbar_wait(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
                 tc_fence_after_sync();
+                GP_MARK(0);
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * kMaxBN;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&full[stage], phase, p.err, 3);
                     tc_fence_after_sync();
+                    GP_MARK(1);
                     const uint32_t sA = smem_u32(stages + (size_t)stage * p.stage_bytes);
                     const uint32_t sB = sA + kABytes;
                     const int k_left = p.K - kb * kBK;
@@ -158,11 +172,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     mma_commit(&empty[stage]);
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+                    GP_MARK(2);
                 }
                 mma_commit(&tmem_full[acc]);
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1;
             }
+            GP_FLUSH(0, 3);
         }
     } else {
         // ------------------------------------------------------------ epilogue
@@ -170,36 +186,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t *my_staging = staging + q * 2 * kStoreBufBytes;
         int acc = 0;
         uint32_t acc_phase = 0, store_idx = 0;
+        GP_DECL;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const int tm = t % p.tiles_m;
             const int tn = (t / p.tiles_m) % p.tiles_n;
             const int b = t / (p.tiles_m * p.tiles_n);
             mbar_wait(&tmem_full[acc], acc_phase, p.err, 4);
             tc_fence_after_sync();
+            GP_MARK(0);
             const int row0 = tm * kBM + q * 32;
             const int row = row0 + lane;
             if (row0 < p.M) {
                 const float rb = (p.row_bias && row < p.M) ? __ldg(p.row_bias + row) : 0.f;
-                for (int chunk = 0; chunk < p.BN / 32; ++chunk) {
+                const int nchunk = min(p.BN / 32, (p.N - tn * p.BN + 31) / 32);
+                const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBN);
+                // one 32x32 block: scale, add, activate, hand to the store path
+                auto finish = [&](const uint32_t (&v)[32], int chunk) {
                     const int col0 = tn * p.BN + chunk * 32;
-                    if (col0 >= p.N) break;
-                    uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBN + chunk * 32), v);
-                    tmem_ld_wait();
                     float f[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float x = p.alpha * __uint_as_float(v[j]) + rb;
-                        if (p.C && row < p.M && col0 + j < p.N)
-                            x = fmaf(p.beta, __ldg(p.C + b * p.c_sb + row * p.c_si + (col0 + j) * p.c_sj), x);
-                        if (p.relu) x = x > 0.f ? x : 0.f;
-                        f[j] = x;
+                    if (p.C == nullptr) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
+                            f[j] = p.relu ? fmaxf(x, 0.f) : x;
+                        }
+                    } else {
+                        // C broadcast: walk one pointer along the row instead of forming 64-bit
+                        // products per element (this branch must stay out of the C-less path)
+                        const float *cp = p.C + b * p.c_sb + (long long)row * p.c_si + (long long)col0 * p.c_sj;
+                        const bool row_ok = row < p.M;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
+                            if (row_ok && col0 + j < p.N) x = fmaf(p.beta, __ldg(cp), x);
+                            cp += p.c_sj;
+                            f[j] = p.relu ? fmaxf(x, 0.f) : x;
+                        }
                     }
+                    GP_MARK(2);
                     if (p.y_tma) {
                         uint8_t *buf = my_staging + (store_idx & 1) * kStoreBufBytes;
                         ++store_idx;
                         if (lane == 0) tma_store_wait_read<1>();   // the store that last read this buffer is done
                         __syncwarp();
+                        GP_MARK(3);
                         // row `lane` of the block, 16-byte chunk c stored at position c ^ (lane % 8)
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
@@ -208,15 +239,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         fence_proxy_async_smem();
                         __syncwarp();
+                        GP_MARK(4);
                         if (lane == 0) {
                             tma_store_3d(&tmY, buf, col0, row0, b);
                             tma_store_commit();
                         }
+                        GP_MARK(5);
                     } else if (row < p.M) {
                         float *yrow = p.Y + b * p.y_sb + (long long)row * p.y_ld;
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             if (col0 + j < p.N) yrow[col0 + j] = f[j];
+                    }
+                };
+                // TMEM reads are software-pipelined: the next block's load is in flight while
+                // the current one is finished and stored
+                uint32_t va[32], vb[32];
+                tmem_ld_32x32(tbase, va);
+                for (int chunk = 0; chunk < nchunk; chunk += 2) {
+                    tmem_ld_wait();
+                    if (chunk + 1 < nchunk) tmem_ld_32x32(tbase + (uint32_t)((chunk + 1) * 32), vb);
+                    GP_MARK(1);
+                    finish(va, chunk);
+                    if (chunk + 1 < nchunk) {
+                        tmem_ld_wait();
+                        if (chunk + 2 < nchunk) tmem_ld_32x32(tbase + (uint32_t)((chunk + 2) * 32), va);
+                        GP_MARK(1);
+                        finish(vb, chunk + 1);
                     }
                 }
             }
@@ -227,6 +276,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (acc == 0) acc_phase ^= 1;
         }
         if (lane == 0) tma_store_wait_all<0>();
+        if (warp == 2 && lane == 0) GP_FLUSH(4, 6);
     }
 
     tc_fence_before_sync();
@@ -310,6 +360,14 @@ int num_sms() {
 }
 
 }  // namespace tc_host
+
+#ifdef ONNXB_PROFILE
+extern "C" int onnxb_dbg_gprofile(long long *out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_gprof, sizeof(long long) * 148 * 16);
+    return 0;
+}
+#endif
 
 bool tc_gemm_supports(const TcGemmProblem &g) {
     if (g.M < 1 || g.N < 1 || g.K < 1 || g.batch < 1) return false;
