@@ -62,7 +62,9 @@ typedef enum {
     ONNXB_KERNEL_SIMT_DIRECT = 0,  /* fp32 FMA direct convolution (thin contractions, any attributes) */
     ONNXB_KERNEL_SIMT_DEPTHWISE = 1, /* fp32 FMA, one input channel per output channel, smem row tiles */
     ONNXB_KERNEL_MMA_GEMM = 2,     /* 1x1 stride-1: batched tcgen05 TF32 GEMM straight from NCHW via TMA */
-    ONNXB_KERNEL_MMA_IMPLICIT = 3  /* general implicit GEMM: TMA staging + in-smem im2col + tcgen05 TF32 */
+    ONNXB_KERNEL_MMA_IMPLICIT = 3, /* general implicit GEMM: TMA staging + in-smem im2col + tcgen05 TF32 */
+    ONNXB_KERNEL_MMA_GATHER_GEMM = 4 /* other 1x1 (strided, or H*W not a multiple of 4): the pixels read are
+                                        gathered into the workspace, then the same batched TF32 GEMM */
 } onnxb_kernel_family;
 
 /*

@@ -17,7 +17,7 @@ OK = 0
 STATUS_NAMES = ["OK", "ERR_NULL", "ERR_ATTR", "ERR_SHAPE", "ERR_UNSUPPORTED", "ERR_WORKSPACE",
                 "ERR_CUDA", "ERR_DEVICE_TIMEOUT"]
 AUTO_PAD = {"NOTSET": 0, "SAME_UPPER": 1, "SAME_LOWER": 2, "VALID": 3}
-KERNEL_FAMILIES = ["simt_direct", "simt_depthwise", "mma_gemm", "mma_implicit"]
+KERNEL_FAMILIES = ["simt_direct", "simt_depthwise", "mma_gemm", "mma_implicit", "mma_gather_gemm"]
 
 EXPORTS = [
     "onnx_conv2d_desc", "onnx_conv2d_desc_query", "onnx_conv2d_desc_query_kernel", "onnx_conv2d_run",

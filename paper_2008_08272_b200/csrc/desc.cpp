@@ -131,6 +131,7 @@ extern "C" onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *a, onnxb_conv
     int family = ONNXB_KERNEL_SIMT_DIRECT;
     if (simt_depthwise_supports(g)) family = ONNXB_KERNEL_SIMT_DEPTHWISE;
     else if (conv_fits_mma_gemm(g)) family = ONNXB_KERNEL_MMA_GEMM;
+    else if (conv_fits_mma_gather_gemm(g)) family = ONNXB_KERNEL_MMA_GATHER_GEMM;
     else if (tc_conv_plan(g, d->plan)) family = ONNXB_KERNEL_MMA_IMPLICIT;
     if (forced == ONNXB_KERNEL_SIMT_DIRECT) family = ONNXB_KERNEL_SIMT_DIRECT;
     else if (forced == ONNXB_KERNEL_SIMT_DEPTHWISE) {
@@ -139,12 +140,17 @@ extern "C" onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *a, onnxb_conv
     } else if (forced == ONNXB_KERNEL_MMA_GEMM) {
         if (!conv_fits_mma_gemm(g)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
         family = ONNXB_KERNEL_MMA_GEMM;
+    } else if (forced == ONNXB_KERNEL_MMA_GATHER_GEMM) {
+        if (!conv_fits_mma_gather_gemm(g)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
+        family = ONNXB_KERNEL_MMA_GATHER_GEMM;
     } else if (forced == ONNXB_KERNEL_MMA_IMPLICIT) {
         if (!tc_conv_plan(g, d->plan, true)) { delete d; return ONNXB_ERR_UNSUPPORTED; }
         family = ONNXB_KERNEL_MMA_IMPLICIT;
     }
     d->family = family;
-    d->workspace_bytes = family == ONNXB_KERNEL_MMA_IMPLICIT ? tc_conv_workspace_bytes(d->plan) : 0;
+    d->workspace_bytes = family == ONNXB_KERNEL_MMA_IMPLICIT     ? tc_conv_workspace_bytes(d->plan)
+                         : family == ONNXB_KERNEL_MMA_GATHER_GEMM ? conv_gather_workspace_bytes(g)
+                                                                  : 0;
     *out = d;
     return ONNXB_OK;
 }

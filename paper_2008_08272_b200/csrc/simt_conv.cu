@@ -3,6 +3,8 @@
 // fallback that accepts every attribute combination of ONNX Conv (Sec. 4.1).
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "common.h"
 
 namespace onnxb {
@@ -137,6 +139,24 @@ conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const flo
     }
 }
 
+// Gather for strided / oddly sized 1x1 convolutions: Xg[plane][j] = X[plane][p*sh][q*sw] for
+// j = p*Q + q < P*Q, zero up to the 16-byte pitch; values rounded to TF32 (nearest, ties away).
+__global__ void __launch_bounds__(256)
+gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, long long total, int pitch, int PQ, int Q,
+                 int HW, int rowstep, int sw) {
+    for (long long i = blockIdx.x * 256LL + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+        const long long plane = i / pitch;
+        const int j = (int)(i - plane * pitch);
+        float v = 0.f;
+        if (j < PQ) {
+            const int p = j / Q, q = j - p * Q;
+            v = __ldg(X + plane * HW + (long long)p * rowstep + q * sw);
+            v = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
+        }
+        Xg[i] = v;
+    }
+}
+
 void depthwise_window(const ConvGeom &g, int &rows, int &cols) {
     rows = (kDwTP - 1) * g.sh + (g.kH - 1) * g.dh + 1;
     cols = (kDwTQ - 1) * g.sw + (g.kW - 1) * g.dw + 1;
@@ -152,6 +172,15 @@ bool simt_depthwise_supports(const ConvGeom &g) {
     if (floats * 4 > 40 * 1024) return false;
     const long long q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;
     return q_tiles * p_tiles * (long long)g.N * g.C <= 2147483647LL;
+}
+
+int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, void *stream) {
+    const long long total = (long long)g.N * g.C * pitch;
+    const long long blocks = std::min<long long>((total + 255) / 256, 148LL * 32);
+    gather1x1_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(X, Xg, total, (int)pitch, g.P * g.Q, g.Q,
+                                                                        g.H * g.W, g.sh * g.W, g.sw);
+    count_launch();
+    return (int)cudaGetLastError();
 }
 
 int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
