@@ -49,20 +49,40 @@ bool conv_fits_mma_gemm(const ConvGeom &g) {
 // of 4 so that TMA cannot address its channel planes): the pixels it reads are first gathered into
 // a dense copy Xg[n][c][pitch] (pitch = P*Q rounded up to 4), rounded to TF32 on the way; then the
 // same GEMM runs on the copy.
-static long long gather_pitch(const ConvGeom &g) { return ((long long)g.P * g.Q + 3) / 4 * 4; }
+// Two layouts of the copy.  Images whose P*Q is a multiple of 4 and not small keep one GEMM per image
+// (Xg[n][c][P*Q], output written by TMA).  Small or oddly sized images are merged: Xg[c][n*P*Q + j]
+// with the row pitch rounded up to 4, so that ONE wide GEMM Y' (M x N*P*Q) = W (M x C) * Xg serves all
+// images and the weights are streamed once per pixel tile instead of once per image; the epilogue then
+// scatters column n*P*Q + j to Y[n][m][j].
+static bool gather_merged(const ConvGeom &g) {
+    const long long PQ = (long long)g.P * g.Q;
+    return PQ % 4 != 0 || PQ < 128;
+}
+static long long gather_pitch(const ConvGeom &g) {
+    const long long PQ = (long long)g.P * g.Q;
+    return gather_merged(g) ? (PQ * g.N + 3) / 4 * 4 : PQ;
+}
 
 static TcGemmProblem conv1x1_gathered_as_gemm(const ConvGeom &g, const float *Xg, const float *W, const float *B,
                                               float *Y) {
     TcGemmProblem t{};
     const long long PQ = (long long)g.P * g.Q, pitch = gather_pitch(g);
-    t.M = g.M; t.N = (int)PQ; t.K = g.C; t.batch = g.N;
+    const bool merged = gather_merged(g);
+    t.M = g.M; t.K = g.C;
     t.A = W; t.B = Xg;
     t.a_mn_major = 0; t.b_mn_major = 1;
-    t.a_ld = g.C; t.b_ld = pitch; t.a_bs = 0; t.b_bs = (long long)g.C * pitch;
-    t.a_batched = 0; t.b_batched = 1;
+    t.a_ld = g.C; t.b_ld = pitch; t.a_bs = 0; t.a_batched = 0;
     t.alpha = 1.f; t.beta = 0.f; t.C = nullptr;
     t.row_bias = B; t.relu = g.relu;
-    t.Y = Y; t.y_ld = PQ; t.y_bs = (long long)g.M * PQ;
+    t.Y = Y; t.y_ld = PQ;
+    if (merged) {
+        t.N = (int)(PQ * g.N); t.batch = 1; t.b_bs = 0; t.b_batched = 0; t.y_bs = 0;
+        t.y_split = (int)PQ; t.y_group_stride = (long long)g.M * PQ;
+    } else {
+        t.N = (int)PQ; t.batch = g.N; t.b_bs = (long long)g.C * pitch; t.b_batched = 1;
+        t.y_bs = (long long)g.M * PQ;
+        t.y_split = 0; t.y_group_stride = 0;
+    }
     return t;
 }
 
@@ -70,11 +90,13 @@ bool conv_fits_mma_gather_gemm(const ConvGeom &g) {
     if (!(g.kH == 1 && g.kW == 1 && g.group == 1)) return false;
     if (g.pt || g.pl || g.pb || g.pr) return false;
     if (g.C < 32) return false;
-    if ((long long)g.N * g.C * gather_pitch(g) > 2147483647LL) return false;
+    if ((long long)g.N * g.C * ((long long)g.P * g.Q + 4) > 2147483647LL) return false;
     return tc_gemm_supports(conv1x1_gathered_as_gemm(g, nullptr, nullptr, nullptr, nullptr));
 }
 
-size_t conv_gather_workspace_bytes(const ConvGeom &g) { return (size_t)g.N * g.C * gather_pitch(g) * 4; }
+size_t conv_gather_workspace_bytes(const ConvGeom &g) {
+    return (size_t)g.C * gather_pitch(g) * 4 * (gather_merged(g) ? 1 : g.N);
+}
 
 }  // namespace onnxb
 
@@ -101,7 +123,8 @@ extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, c
             err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y), cuda_stream);
             break;
         case ONNXB_KERNEL_MMA_GATHER_GEMM:
-            err = launch_gather1x1(d->g, X, static_cast<float *>(workspace), gather_pitch(d->g), cuda_stream);
+            err = launch_gather1x1(d->g, X, static_cast<float *>(workspace), gather_pitch(d->g), gather_merged(d->g),
+                                   cuda_stream);
             if (err == 0)
                 err = launch_tc_gemm(conv1x1_gathered_as_gemm(d->g, static_cast<const float *>(workspace), W, B, Y),
                                      cuda_stream);

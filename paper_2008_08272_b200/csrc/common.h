@@ -47,7 +47,7 @@ bool simt_depthwise_supports(const ConvGeom &g);
 bool conv_fits_mma_gemm(const ConvGeom &g);
 bool conv_fits_mma_gather_gemm(const ConvGeom &g);   // other unpadded 1x1: gather the pixels read, then the same GEMM
 size_t conv_gather_workspace_bytes(const ConvGeom &g);
-int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, void *stream);
+int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, bool merged, void *stream);
 // implicit-GEMM tensor-core convolution (tc_conv.cu)
 bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan, bool forced = false);
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan);

@@ -139,17 +139,28 @@ conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const flo
     }
 }
 
-// Gather for strided / oddly sized 1x1 convolutions: Xg[plane][j] = X[plane][p*sh][q*sw] for
-// j = p*Q + q < P*Q, zero up to the 16-byte pitch; values rounded to TF32 (nearest, ties away).
+// Gather for strided / oddly sized 1x1 convolutions, values rounded to TF32 (nearest, ties away):
+//   merged:    Xg[c][n*P*Q + p*Q + q] = X[n][c][p*sh][q*sw], rows padded with zeros to the pitch;
+//   per image: Xg[n][c][p*Q + q]      (pitch = P*Q).
 __global__ void __launch_bounds__(256)
-gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, long long total, int pitch, int PQ, int Q,
-                 int HW, int rowstep, int sw) {
+gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, long long total, int pitch, int NPQ, int PQ,
+                 int Q, int C, int HW, int rowstep, int sw, int merged) {
     for (long long i = blockIdx.x * 256LL + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
-        const long long plane = i / pitch;
-        const int j = (int)(i - plane * pitch);
+        const long long row = i / pitch;              // merged: channel; per image: n*C + c
+        const int j = (int)(i - row * pitch);
         float v = 0.f;
-        if (j < PQ) {
-            const int p = j / Q, q = j - p * Q;
+        if (j < NPQ) {
+            long long plane;
+            int r;
+            if (merged) {
+                const int n = j / PQ;
+                r = j - n * PQ;
+                plane = (long long)n * C + row;
+            } else {
+                r = j;
+                plane = row;
+            }
+            const int p = r / Q, q = r - p * Q;
             v = __ldg(X + plane * HW + (long long)p * rowstep + q * sw);
             v = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
         }
@@ -174,11 +185,12 @@ bool simt_depthwise_supports(const ConvGeom &g) {
     return q_tiles * p_tiles * (long long)g.N * g.C <= 2147483647LL;
 }
 
-int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, void *stream) {
-    const long long total = (long long)g.N * g.C * pitch;
+int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, bool merged, void *stream) {
+    const long long total = merged ? (long long)g.C * pitch : (long long)g.N * g.C * pitch;
     const long long blocks = std::min<long long>((total + 255) / 256, 148LL * 32);
-    gather1x1_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(X, Xg, total, (int)pitch, g.P * g.Q, g.Q,
-                                                                        g.H * g.W, g.sh * g.W, g.sw);
+    gather1x1_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
+        X, Xg, total, (int)pitch, merged ? g.N * g.P * g.Q : g.P * g.Q, g.P * g.Q, g.Q, g.C, g.H * g.W, g.sh * g.W,
+        g.sw, merged ? 1 : 0);
     count_launch();
     return (int)cudaGetLastError();
 }

@@ -65,6 +65,8 @@ struct Params {
     int relu;
     float *Y;                  // used by the plain-store epilogue
     long long y_ld, y_sb;
+    int y_split;               // > 0: columns are groups of y_split, y_group elements apart (plain stores only)
+    long long y_group;
     int y_tma;
     unsigned int *err;
 };
@@ -204,7 +206,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 auto finish = [&](const uint32_t (&v)[32], int chunk) {
                     const int col0 = tn * p.BN + chunk * 32;
                     float f[32];
-#pragma unroll
                     if (p.C == nullptr) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
@@ -225,18 +226,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                     GP_MARK(2);
+                    // Stage the 32x32 block in shared memory, row `lane`, 16-byte chunk c at position
+                    // c ^ (lane % 8) (the 128-byte swizzle, conflict-free for these 16-byte stores).
+                    uint8_t *buf = my_staging + (store_idx & 1) * kStoreBufBytes;
+                    ++store_idx;
                     if (p.y_tma) {
-                        uint8_t *buf = my_staging + (store_idx & 1) * kStoreBufBytes;
-                        ++store_idx;
                         if (lane == 0) tma_store_wait_read<1>();   // the store that last read this buffer is done
-                        __syncwarp();
-                        GP_MARK(3);
-                        // row `lane` of the block, 16-byte chunk c stored at position c ^ (lane % 8)
+                    }
+                    __syncwarp();
+                    GP_MARK(3);
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            float4 val = make_float4(f[4 * c], f[4 * c + 1], f[4 * c + 2], f[4 * c + 3]);
-                            *reinterpret_cast<float4 *>(buf + lane * 128 + ((c ^ (lane & 7)) << 4)) = val;
-                        }
+                    for (int c = 0; c < 8; ++c) {
+                        float4 val = make_float4(f[4 * c], f[4 * c + 1], f[4 * c + 2], f[4 * c + 3]);
+                        *reinterpret_cast<float4 *>(buf + lane * 128 + ((c ^ (lane & 7)) << 4)) = val;
+                    }
+                    if (p.y_tma) {
                         fence_proxy_async_smem();
                         __syncwarp();
                         GP_MARK(4);
@@ -245,11 +249,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             tma_store_commit();
                         }
                         GP_MARK(5);
-                    } else if (row < p.M) {
-                        float *yrow = p.Y + b * p.y_sb + (long long)row * p.y_ld;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) yrow[col0 + j] = f[j];
+                    } else {
+                        // Y rows cannot be described to TMA (row pitch not a multiple of 16 bytes): read the
+                        // block back transposed, lanes along the columns, and store row by row (coalesced).
+                        __syncwarp();
+                        const int col = col0 + lane;
+                        const int rows = min(32, p.M - row0);
+                        long long coff = col;
+                        if (p.y_split > 0) {
+                            const int grp = col / p.y_split;
+                            coff = (long long)grp * p.y_group + (col - grp * p.y_split);
+                        }
+                        float *yp = p.Y + b * p.y_sb + (long long)row0 * p.y_ld + coff;
+                        for (int r = 0; r < rows; ++r) {
+                            const float val = *reinterpret_cast<const float *>(
+                                buf + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2)));
+                            if (col < p.N) *yp = val;
+                            yp += p.y_ld;
+                        }
+                        __syncwarp();
                     }
                 };
                 // TMEM reads are software-pipelined: the next block's load is in flight while
@@ -398,7 +416,8 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
     p.row_bias = g.row_bias; p.relu = g.relu;
     p.Y = g.Y; p.y_ld = g.y_ld; p.y_sb = g.y_bs;
-    p.y_tma = (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);
+    p.y_split = g.y_split; p.y_group = g.y_group_stride;
+    p.y_tma = g.y_split == 0 && (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);
     p.err = device_status_ptr();
     if (!p.err) return (int)cudaErrorUnknown;
 

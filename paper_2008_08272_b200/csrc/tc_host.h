@@ -23,6 +23,11 @@ struct TcGemmProblem {
     int relu;
     float *Y;
     long long y_ld, y_bs;
+    // When y_split > 0 the N columns are `y_split`-wide groups laid y_group_stride elements apart in Y
+    // (column j lives at (j / y_split) * y_group_stride + j % y_split of its row): the pixels of several
+    // NCHW images contracted as one wide GEMM.
+    int y_split;
+    long long y_group_stride;
 };
 
 bool tc_gemm_supports(const TcGemmProblem &g);
