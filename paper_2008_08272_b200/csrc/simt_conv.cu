@@ -93,17 +93,19 @@ conv2d_direct_kernel(const ConvGeom g, const float *__restrict__ X, const float 
 }
 
 // Depthwise convolution (group == C == M): purely HBM-bound, 2*kH*kW flops per
-// output.  A block stages the input window of a TP x TQ output tile of one
+// output.  A block stages the input window of a 32 x 32 output tile of one
 // (image, channel) plane in shared memory with coalesced row loads (zeros
-// outside the image), then every thread produces one output from shared memory.
-constexpr int kDwTP = 8, kDwTQ = 32;
+// outside the image); each of its 256 threads then produces a column strip of
+// four vertically adjacent outputs, so the rows of the window shared by the
+// four outputs are read from shared memory once per tap column.
+constexpr int kDwTP = 32, kDwTQ = 32, kDwRows = 4, kDwThreads = kDwTQ * (kDwTP / kDwRows);
 
-__global__ void __launch_bounds__(kDwTP *kDwTQ)
+__global__ void __launch_bounds__(kDwThreads)
 conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
                         const float *__restrict__ B, float *__restrict__ Y, int q_tiles, int p_tiles,
-                        int in_rows, int in_cols) {
-    extern __shared__ float tile[];           // [in_rows][in_cols] then weights [kH*kW]
-    float *wsm = tile + in_rows * in_cols;
+                        int in_rows, int in_cols, int pitch) {
+    extern __shared__ float tile[];           // [in_rows][pitch] then weights [kH*kW]
+    float *wsm = tile + in_rows * pitch;
 
     int bid = blockIdx.x;
     const int qt = bid % q_tiles; bid /= q_tiles;
@@ -115,27 +117,43 @@ conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const flo
     const float *xp = X + (size_t)plane * g.H * g.W;
 
     const int taps = g.kH * g.kW;
-    for (int i = threadIdx.x; i < taps; i += blockDim.x) wsm[i] = W[(size_t)c * taps + i];
-    for (int i = threadIdx.x; i < in_rows * in_cols; i += blockDim.x) {
+    for (int i = threadIdx.x; i < taps; i += kDwThreads) wsm[i] = W[(size_t)c * taps + i];
+    // window rows actually needed by this tile (fewer at the bottom edge of the image)
+    const int rows_out = min(kDwTP, g.P - p0);
+    const int rows_in = min(in_rows, (rows_out - 1) * g.sh + (g.kH - 1) * g.dh + 1);
+    for (int i = threadIdx.x; i < rows_in * in_cols; i += kDwThreads) {
         const int rr = i / in_cols, cc = i - rr * in_cols;
         const int ih = ih0 + rr, iw = iw0 + cc;
         float v = 0.f;
         if ((unsigned)ih < (unsigned)g.H && (unsigned)iw < (unsigned)g.W) v = __ldg(xp + (size_t)ih * g.W + iw);
-        tile[i] = v;
+        tile[rr * pitch + cc] = v;
     }
     __syncthreads();
 
-    const int tq = threadIdx.x % kDwTQ, tp = threadIdx.x / kDwTQ;
-    const int p = p0 + tp, q = q0 + tq;
-    if (p < g.P && q < g.Q) {
-        float acc = 0.f;
+    const int tq = threadIdx.x % kDwTQ, tp = (threadIdx.x / kDwTQ) * kDwRows;
+    const int q = q0 + tq;
+    if (q >= g.Q || p0 + tp >= g.P) return;
+    float acc[kDwRows];
+#pragma unroll
+    for (int k = 0; k < kDwRows; ++k) acc[k] = 0.f;
+    for (int s = 0; s < g.kW; ++s) {
+        const float *col = tile + tq * g.sw + s * g.dw;
         for (int r = 0; r < g.kH; ++r) {
-            const float *row = tile + (tp * g.sh + r * g.dh) * in_cols + tq * g.sw;
-            for (int s = 0; s < g.kW; ++s) acc = fmaf(row[s * g.dw], wsm[r * g.kW + s], acc);
+            const float w = wsm[r * g.kW + s];
+#pragma unroll
+            for (int k = 0; k < kDwRows; ++k)
+                if (tp + k < rows_out) acc[k] = fmaf(col[((tp + k) * g.sh + r * g.dh) * pitch], w, acc[k]);
         }
-        acc += B ? __ldg(B + c) : 0.f;
-        if (g.relu) acc = acc > 0.f ? acc : 0.f;
-        Y[((size_t)plane * g.P + p) * g.Q + q] = acc;
+    }
+    const float bias = B ? __ldg(B + c) : 0.f;
+#pragma unroll
+    for (int k = 0; k < kDwRows; ++k) {
+        const int p = p0 + tp + k;
+        if (p < g.P) {
+            float v = acc[k] + bias;
+            if (g.relu) v = v > 0.f ? v : 0.f;
+            Y[((size_t)plane * g.P + p) * g.Q + q] = v;
+        }
     }
 }
 
@@ -168,19 +186,20 @@ gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, long long 
     }
 }
 
-void depthwise_window(const ConvGeom &g, int &rows, int &cols) {
+void depthwise_window(const ConvGeom &g, int &rows, int &cols, int &pitch) {
     rows = (kDwTP - 1) * g.sh + (g.kH - 1) * g.dh + 1;
     cols = (kDwTQ - 1) * g.sw + (g.kW - 1) * g.dw + 1;
+    pitch = cols | 1;                          // odd pitch: strided column reads stay conflict-free
 }
 
 }  // namespace
 
 bool simt_depthwise_supports(const ConvGeom &g) {
     if (!(g.Cg == 1 && g.Mg == 1)) return false;
-    int rows, cols;
-    depthwise_window(g, rows, cols);
-    const long long floats = (long long)rows * cols + (long long)g.kH * g.kW;
-    if (floats * 4 > 40 * 1024) return false;
+    int rows, cols, pitch;
+    depthwise_window(g, rows, cols, pitch);
+    const long long floats = (long long)rows * pitch + (long long)g.kH * g.kW;
+    if (floats * 4 > 96 * 1024) return false;
     const long long q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;
     return q_tiles * p_tiles * (long long)g.N * g.C <= 2147483647LL;
 }
@@ -197,13 +216,18 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
 
 int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
                           void *stream) {
-    int rows, cols;
-    depthwise_window(g, rows, cols);
+    int rows, cols, pitch;
+    depthwise_window(g, rows, cols, pitch);
     const int q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;
-    const size_t smem = ((size_t)rows * cols + (size_t)g.kH * g.kW) * sizeof(float);
+    const size_t smem = ((size_t)rows * pitch + (size_t)g.kH * g.kW) * sizeof(float);
+    if (smem > 48 * 1024) {
+        const cudaError_t e =
+            cudaFuncSetAttribute(conv2d_depthwise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        if (e != cudaSuccess) return (int)e;
+    }
     const unsigned blocks = (unsigned)((long long)q_tiles * p_tiles * g.N * g.C);
-    conv2d_depthwise_kernel<<<blocks, kDwTP * kDwTQ, smem, (cudaStream_t)stream>>>(g, X, W, B, Y, q_tiles, p_tiles,
-                                                                                 rows, cols);
+    conv2d_depthwise_kernel<<<blocks, kDwThreads, smem, (cudaStream_t)stream>>>(g, X, W, B, Y, q_tiles, p_tiles, rows,
+                                                                              cols, pitch);
     count_launch();
     return (int)cudaGetLastError();
 }
