@@ -160,29 +160,53 @@ conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const flo
 // Gather for strided / oddly sized 1x1 convolutions, values rounded to TF32 (nearest, ties away):
 //   merged:    Xg[c][n*P*Q + p*Q + q] = X[n][c][p*sh][q*sw], rows padded with zeros to the pitch;
 //   per image: Xg[n][c][p*Q + q]      (pitch = P*Q).
+__device__ __forceinline__ float gather_round(float v) {
+    return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
+}
+
 __global__ void __launch_bounds__(256)
-gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, long long total, int pitch, int NPQ, int PQ,
-                 int Q, int C, int HW, int rowstep, int sw, int merged) {
-    for (long long i = blockIdx.x * 256LL + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
-        const long long row = i / pitch;              // merged: channel; per image: n*C + c
-        const int j = (int)(i - row * pitch);
+gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, unsigned total, unsigned pitch, unsigned NPQ,
+                 unsigned PQ, unsigned Q, unsigned C, unsigned HW, unsigned rowstep, unsigned sw, int merged) {
+    for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total; i += gridDim.x * 256u) {
+        const unsigned row = i / pitch;               // merged: channel; per image: n*C + c
+        const unsigned j = i - row * pitch;
         float v = 0.f;
         if (j < NPQ) {
-            long long plane;
-            int r;
+            unsigned plane, r;
             if (merged) {
-                const int n = j / PQ;
+                const unsigned n = j / PQ;
                 r = j - n * PQ;
-                plane = (long long)n * C + row;
+                plane = n * C + row;
             } else {
                 r = j;
                 plane = row;
             }
-            const int p = r / Q, q = r - p * Q;
-            v = __ldg(X + plane * HW + (long long)p * rowstep + q * sw);
-            v = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
+            const unsigned p = r / Q, q = r - p * Q;
+            v = gather_round(__ldg(X + (size_t)plane * HW + p * rowstep + q * sw));
         }
         Xg[i] = v;
+    }
+}
+
+// Per-image layout, Q a multiple of 4, W a multiple of 4, column stride 1 or 2: four outputs per
+// thread from one or two aligned 16-byte loads, one 16-byte store.
+template <int SW>
+__global__ void __launch_bounds__(256)
+gather1x1_vec_kernel(const float4 *__restrict__ X4, float4 *__restrict__ Xg4, unsigned total4, unsigned PQ4,
+                     unsigned Q4, unsigned HW4, unsigned rowstep4) {
+    for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total4; i += gridDim.x * 256u) {
+        const unsigned plane = i / PQ4, r = i - plane * PQ4;
+        const unsigned p = r / Q4, q4 = r - p * Q4;
+        const float4 *src = X4 + (size_t)plane * HW4 + p * rowstep4 + q4 * SW;
+        float4 o;
+        if (SW == 1) {
+            o = __ldg(src);
+        } else {
+            const float4 a = __ldg(src), b = __ldg(src + 1);
+            o = make_float4(a.x, a.z, b.x, b.z);
+        }
+        o.x = gather_round(o.x); o.y = gather_round(o.y); o.z = gather_round(o.z); o.w = gather_round(o.w);
+        Xg4[i] = o;
     }
 }
 
@@ -206,10 +230,26 @@ bool simt_depthwise_supports(const ConvGeom &g) {
 
 int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pitch, bool merged, void *stream) {
     const long long total = merged ? (long long)g.C * pitch : (long long)g.N * g.C * pitch;
-    const long long blocks = std::min<long long>((total + 255) / 256, 148LL * 32);
-    gather1x1_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
-        X, Xg, total, (int)pitch, merged ? g.N * g.P * g.Q : g.P * g.Q, g.P * g.Q, g.Q, g.C, g.H * g.W, g.sh * g.W,
-        g.sw, merged ? 1 : 0);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!merged && g.Q % 4 == 0 && g.W % 4 == 0 && (g.sw == 1 || g.sw == 2) && g.Q * g.sw <= g.W) {
+        const long long total4 = total / 4;
+        const unsigned blocks = (unsigned)std::min<long long>((total4 + 255) / 256, 148LL * 16);
+        const unsigned PQ4 = g.P * g.Q / 4, Q4 = g.Q / 4, HW4 = g.H * g.W / 4, rowstep4 = g.sh * g.W / 4;
+        if (g.sw == 1)
+            gather1x1_vec_kernel<1><<<blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(X),
+                                                           reinterpret_cast<float4 *>(Xg), (unsigned)total4, PQ4, Q4,
+                                                           HW4, rowstep4);
+        else
+            gather1x1_vec_kernel<2><<<blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(X),
+                                                           reinterpret_cast<float4 *>(Xg), (unsigned)total4, PQ4, Q4,
+                                                           HW4, rowstep4);
+    } else {
+        const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, 148LL * 32);
+        gather1x1_kernel<<<blocks, 256, 0, st>>>(X, Xg, (unsigned)total, (unsigned)pitch,
+                                                 (unsigned)(merged ? g.N * g.P * g.Q : g.P * g.Q), (unsigned)(g.P * g.Q),
+                                                 (unsigned)g.Q, (unsigned)g.C, (unsigned)(g.H * g.W),
+                                                 (unsigned)(g.sh * g.W), (unsigned)g.sw, merged ? 1 : 0);
+    }
     count_launch();
     return (int)cudaGetLastError();
 }
