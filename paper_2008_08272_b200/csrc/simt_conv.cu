@@ -6,6 +6,7 @@
 #include <algorithm>
 
 #include "common.h"
+#include "tc_common.cuh"
 
 namespace onnxb {
 
@@ -167,6 +168,7 @@ __device__ __forceinline__ float gather_round(float v) {
 __global__ void __launch_bounds__(256)
 gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, unsigned total, unsigned pitch, unsigned NPQ,
                  unsigned PQ, unsigned Q, unsigned C, unsigned HW, unsigned rowstep, unsigned sw, int merged) {
+    tc::pdl_launch_dependents();
     for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total; i += gridDim.x * 256u) {
         const unsigned row = i / pitch;               // merged: channel; per image: n*C + c
         const unsigned j = i - row * pitch;
@@ -194,6 +196,7 @@ template <int SW>
 __global__ void __launch_bounds__(256)
 gather1x1_vec_kernel(const float4 *__restrict__ X4, float4 *__restrict__ Xg4, unsigned total4, unsigned PQ4,
                      unsigned Q4, unsigned HW4, unsigned rowstep4) {
+    tc::pdl_launch_dependents();
     for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total4; i += gridDim.x * 256u) {
         const unsigned plane = i / PQ4, r = i - plane * PQ4;
         const unsigned p = r / Q4, q4 = r - p * Q4;

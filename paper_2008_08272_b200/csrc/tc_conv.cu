@@ -85,6 +85,7 @@ __device__ long long g_chk[8];
 // terms each) per output channel, rows 16 bytes apart.  Values are rounded to TF32 (nearest);
 // rows past the group's channels, channels past Cg and unpaired taps are zero.
 __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict__ W, float4 *__restrict__ out) {
+    pdl_launch_dependents();
     const long long total = g.packed_floats / 4;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -155,6 +156,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_holder;
+    pdl_launch_dependents();
+    pdl_wait();                 // everything above overlapped the previous kernel's tail
 
     if (warp == 0) {
         // ------------------------------------------------------------ raw activation producer
@@ -743,9 +746,10 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
             plan.n_steps, plan.spb, plan.total_tiles, grid, plan.raw_mode, plan.BOXP, plan.a_stage_bytes,
             plan.raw_stage_bytes, plan.b_stage_bytes, plan.nb_stages, smem);
 #endif
-    tc_conv_kernel<<<grid, kThreads, smem, st>>>(tmX, plan, X, reinterpret_cast<const float *>(workspace), B, Y, err);
+    const cudaError_t le = launch_pdl(tc_conv_kernel, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+                                      reinterpret_cast<const float *>(workspace), B, Y, err);
     count_launch();
-    return (int)cudaGetLastError();
+    return (int)le;
 }
 
 }  // namespace onnxb

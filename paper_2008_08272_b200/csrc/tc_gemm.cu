@@ -110,6 +110,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
+    pdl_launch_dependents();
+    pdl_wait();                 // everything above overlapped the previous kernel's tail
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -464,9 +466,10 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     if (attr_err != cudaSuccess) return (int)attr_err;
     const long long total = (long long)p.tiles_m * p.tiles_n * p.batch;
     const int grid = (int)(total < sms ? total : sms);
-    tc_gemm_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(tmA, tmB, tmY, p);
+    const cudaError_t le = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB,
+                                      tmY, p);
     count_launch();
-    return (int)cudaGetLastError();
+    return (int)le;
 }
 
 }  // namespace onnxb
