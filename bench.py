@@ -204,7 +204,12 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     binding.load(build_if_missing=False)
 
-    convs, gemm = step_ops()
+    convs, gemm = step_ops(args.batch)
+    if args.only:
+        # profiling aid: a subset of the step's convolutions (name substring), e.g. one layer under ncu
+        convs = [c for c in convs if args.only in c.name]
+        if not convs:
+            raise SystemExit(f"--only {args.only!r} matches no convolution of the step")
     # ---- inputs: seeded host arrays (pinned, reused by the e2e leg) and resident device copies
     host, devt, descs = [], [], []
     for c in convs:
@@ -385,7 +390,9 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "tf32" if any(f.startswith("mma") for f in families) else "f32",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "batch_per_gpu": 64, "ops_per_step": n_ops,
+        "config": {"workload": WORKLOAD if not args.only and args.batch == 64 else
+                   f"SUBSET only={args.only!r} batch={args.batch} (profiling aid, not the benchmark)",
+                   "batch_per_gpu": args.batch, "ops_per_step": n_ops,
                    "gflop_per_step": round(flops_per_step / 1e9, 3),
                    "l2": "inputs larger than L2: every op has its own X/W/Y buffers, ~8 GB touched per step",
                    "parallelism": f"replicas x{world} (batch split, no collective)"},
@@ -406,6 +413,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="", help="profiling aid: run only the convolutions whose name contains this")
+    ap.add_argument("--batch", type=int, default=64, help="images per convolution (the benchmark proper uses 64)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
