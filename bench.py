@@ -29,9 +29,33 @@ from paper_2008_08272_b200 import workloads as wl  # noqa: E402
 METRIC = "Conv/Gemm TFLOP/s (fp32 I/O, TF32 MMA)"
 WORKLOAD = "resnet50_v1_53conv_sweep_b64+depthwise_256x28x28+gemm_head_64x1000x2048"
 TF32_OVER_BF16 = 1125.0 / 2250.0     # nominal dense ratio, applied to the measured bf16 peak
-SAMPLE_IMAGES = 4
-SAMPLE_TEXT = ("first 4 images of each of the 54 convolutions plus the full head Gemm "
-               "(1/16 of a step's convolution work)")
+SAMPLE_IMAGES = 16
+SAMPLE_TEXT = ("first 16 images of each of the 54 convolutions plus the full head Gemm "
+               "(1/4 of a step's convolution work)")
+
+# DRAM traffic of the implicit-GEMM convolution kernel per benchmark step (its 17 launches), from the
+# ncu captures summarised in profiles/tc_conv_kernel_dram_traffic_per_layer_shape.md.  Valid only for
+# the kernel source those captures ran: the hash below is checked at run time.
+NCU_TRAFFIC = {"mma_implicit": {"bytes_per_step": 599.3e6,
+                                "sources": ["paper_2008_08272_b200/csrc/tc_conv.cu",
+                                            "paper_2008_08272_b200/csrc/tc_conv_plan.h"],
+                                "sha1": "20475de901e83c6c46367ed851a9e22c30156af4"}}
+
+
+def ncu_traffic(family):
+    """Measured DRAM bytes per step for `family`, or None when no capture matches the current source."""
+    import hashlib
+    rec = NCU_TRAFFIC.get(family)
+    if rec is None:
+        return None
+    h = hashlib.sha1()
+    try:
+        for f in rec["sources"]:
+            with open(os.path.join(ROOT, f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return rec["bytes_per_step"] if h.hexdigest() == rec["sha1"] else None
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max clock
 
 
@@ -320,8 +344,10 @@ def run_ours(args):
         roof = {"bound": "alu", "achieved": ach_tflops, "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s",
                 "frac": ach_tflops / FP32_FMA_PEAK_TFLOPS,
                 "peak_source": "derived: 148 SMs x 128 fp32 FMA/clk x 2 x 1.965 GHz"}
+    only_full = (not args.only) and args.batch == 64
     roof.update({"kernel": top, "launches_per_step": fam_count[top], "ms_per_step": fam_time[top],
-                 "traffic": None})
+                 "basis": "all launches of this kernel family in one step (flops or bytes summed, time summed)",
+                 "traffic": ncu_traffic(top) if only_full else None, "traffic_unit": "bytes per step"})
     families_out = {f: {"ops": fam_count[f], "ms": round(fam_time[f], 4),
                         "tflops": round(fam_flops[f] / (fam_time[f] * 1e-3) / 1e12, 3),
                         "gbs": round(fam_bytes[f] / (fam_time[f] * 1e-3) / 1e9, 1)} for f in fam_time}
