@@ -12,8 +12,15 @@
 //   warp 2      issues, for every tap, tcgen05.mma on the SAME activation tile at a start address
 //               shifted by the tap's slot offset, accumulating in TMEM;
 //   warps 11-18 read finished accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
-//               with lanes along consecutive pixels (coalesced); with one 128-row accumulator per
-//               tile TMEM holds two of them, so this overlaps the next tile's MMAs.
+//               with lanes along consecutive pixels (coalesced); when a tile's accumulators fill at
+//               most half of TMEM it holds two sets, so this overlaps the next tile's MMAs.
+// CTA pairs (kCtas = 2): two CTAs of a cluster share one tile of 2 x MT x 128 pixels.  Each stages
+// its own pixels and HALF of the tile's weight rows; the even CTA issues cta_group::2 MMAs
+// (M = 256) that read both CTAs' shared memory and write each CTA's rows into its own TMEM.  Per
+// CTA this halves the weight bytes fetched from L2 and the weight bytes the tensor pipe reads from
+// shared memory per flop, the two limits of the single-CTA form.  Stage hand-over: the odd CTA's
+// transform and epilogue warps arrive directly on the even CTA's barriers, its MMA warp forwards
+// "my weights have landed", and stage releases come back by multicast commit.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -37,7 +44,9 @@ constexpr int kThreads = 608;              // 19 warps: 2 producers, MMA, 8 tran
 constexpr int kXformWarps = 8;
 constexpr int kXformThreads = kXformWarps * 32;
 constexpr int kEpiWarps = 8;
-constexpr int kOwned = 10;                 // slots of an A stage one transform thread may own
+constexpr int kOwned = 10;                 // (slot, chunk) units of an A stage one transform thread may own
+constexpr int kMaxRawStages = 4;
+constexpr int kMaxSpb = 8;                 // K-steps per weight stage (the MMA issue loop is unrolled over them)
 constexpr int kMaxBStages = 12;
 constexpr int kSmemLimit = 232448;
 constexpr int kBarBytes = 512;
@@ -45,9 +54,10 @@ constexpr int kSegBytes = 256;             // >= sizeof(TcConvSegs)
 static_assert(sizeof(TcConvSegs) <= kSegBytes, "segment table does not fit its slot");
 
 struct Bars {
-    uint64_t raw_full[2], raw_empty[2], a_full[2], a_empty[2];
+    uint64_t raw_full[kMaxRawStages], raw_empty[kMaxRawStages], a_full[2], a_empty[2];
     uint64_t b_full[kMaxBStages], b_empty[kMaxBStages];
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t seg_full[2], seg_empty[2];      // segment tables, one per tile parity
     uint32_t tmem_holder;
 };
 static_assert(sizeof(Bars) <= kBarBytes, "barrier block too large");
@@ -58,7 +68,11 @@ __device__ long long g_prof[148 * 16];
 #define PROF_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
 #define PROF_RESET() do { pt_ = clock64(); } while (0)
 #define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 5; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
+// event log of CTA 0: kind k (0..7), sequence number i (0..63) -> clock
+__device__ long long g_log[8 * 64];
+#define LOG(k, i) do { if (blockIdx.x == 0 && (i) < 64) g_log[(k) * 64 + (i)] = clock64(); } while (0)
 #else
+#define LOG(k, i) do {} while (0)
 #define PROF_DECL do {} while (0)
 #define PROF_MARK(k) do {} while (0)
 #define PROF_RESET() do {} while (0)
@@ -80,9 +94,9 @@ __device__ long long g_chk[8];
 #endif
 
 // ------------------------------------------------------------------ weight packing
-// Packed layout: [group][channel tile][channel block][K-step][chunk 0/1][row BN][4], i.e. for each
-// K-step the exact shared-memory image of the K-major B operand: two 16-byte chunks (4 reduction
-// terms each) per output channel, rows 16 bytes apart.  Values are rounded to TF32 (nearest);
+// Packed layout: [group][channel tile][CTA of the pair][channel block][K-step][chunk 0/1][row BNH][4],
+// i.e. for each K-step the exact shared-memory image of one CTA's part of the K-major B operand: two
+// 16-byte chunks (4 reduction terms each) per output channel, rows 16 bytes apart.  Values are rounded to TF32 (nearest);
 // rows past the group's channels, channels past Cg and unpaired taps are zero.
 __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict__ W, float4 *__restrict__ out) {
     pdl_launch_dependents();
@@ -90,13 +104,13 @@ __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict_
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
         long long t = i;
-        const int row = (int)(t % g.BN); t /= g.BN;
+        const int row = (int)(t % g.BNH); t /= g.BNH;
         const int k = (int)(t % 2); t /= 2;
         const int step = (int)(t % g.n_steps); t /= g.n_steps;
         const int cb = (int)(t % g.ncb); t /= g.ncb;
-        const int ct = (int)(t % g.ctiles); t /= g.ctiles;
+        const int ct = (int)(t % (g.ctiles * g.ctas)); t /= g.ctiles * g.ctas;   // BNH-wide tile: (tile, CTA of the pair)
         const int grp = (int)t;
-        const int mg = ct * g.BN + row;
+        const int mg = ct * g.BNH + row;
         const int tap = g.src_tap[step][k];
         float v[4] = {0.f, 0.f, 0.f, 0.f};
         if (mg < g.Mg && tap >= 0) {
@@ -112,7 +126,13 @@ __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict_
     }
 }
 
+// Channel blocks are summed in a rotated order that differs from tile to tile: CTAs working at the
+// same time then stream different parts of the (shared) packed weights, instead of all asking the
+// same L2 lines at the same moment.
+__device__ __forceinline__ int cb_rotation(long long tile, int ncb) { return (int)((tile * 5 + 3) % ncb); }
+
 // ------------------------------------------------------------------ main kernel
+template <int kCtas>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, const float *__restrict__ X,
                const float *__restrict__ Wpk, const float *__restrict__ bias, float *__restrict__ Y,
@@ -123,27 +143,39 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *a_st = smem;
     uint8_t *raw_st = a_st + 2 * (size_t)g.a_stage_bytes;
-    uint8_t *b_st = raw_st + 2 * (size_t)g.raw_stage_bytes;
+    uint8_t *b_st = raw_st + (size_t)g.nr_stages * g.raw_stage_bytes;
     uint8_t *seg_st = b_st + (size_t)g.nb_stages * g.b_stage_bytes;
-    Bars *bars = reinterpret_cast<Bars *>(seg_st + 2 * kSegBytes);
+    Bars *bars = reinterpret_cast<Bars *>(seg_st + kMaxRawStages * kSegBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile_rows = g.MT * 128;
+    // CTA pair: rank within the cluster, and the tiles this CTA (pair) walks
+    const uint32_t rank = kCtas == 2 ? cluster_ctarank() : 0u;
+    const long long first_tile = blockIdx.x / kCtas, tile_step = gridDim.x / kCtas;
+    const int cgt = g.ctiles * g.group;        // channel tiles over all groups
+    // accumulator placement in TMEM: two alternating sets when one set fits in 256 columns
+    const bool acc_dbl = g.MT == 1 || g.BN <= 128;
+    const uint32_t mt_cols = acc_dbl ? 128u : 256u;     // column distance between a CTA's two accumulators
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < g.nr_stages; ++s) {
             mbar_init(&bars->raw_full[s], 1);
             mbar_init(&bars->raw_empty[s], kXformWarps);
-            mbar_init(&bars->a_full[s], kXformWarps);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->a_full[s], kXformWarps * kCtas);      // waited on by the issuing CTA only
             mbar_init(&bars->a_empty[s], 1);
         }
         for (int s = 0; s < g.nb_stages; ++s) {
-            mbar_init(&bars->b_full[s], 1);
+            // issuing CTA of a pair: its own producer plus the peer's "landed" message
+            mbar_init(&bars->b_full[s], (kCtas == 2 && rank == 0) ? 2 : 1);
             mbar_init(&bars->b_empty[s], 1);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->acc_full[s], 1);
-            mbar_init(&bars->acc_empty[s], kEpiWarps);
+            mbar_init(&bars->acc_empty[s], kEpiWarps * kCtas);
+            mbar_init(&bars->seg_full[s], 1);
+            mbar_init(&bars->seg_empty[s], kXformWarps);
         }
         mbar_fence_init();
         if (g.raw_mode == 0) prefetch_tmap(&tmX);
@@ -156,6 +188,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_holder;
+    if (kCtas == 2) cluster_sync_all();     // the peer's barriers exist before anything arrives on them
     pdl_launch_dependents();
     pdl_wait();                 // everything above overlapped the previous kernel's tail
 
@@ -163,31 +196,32 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         // ------------------------------------------------------------ raw activation producer
         if (elect_one()) {
             int rs = 0;
-            uint32_t rphase = 0;
+            uint32_t rphase = 0, tile_it = 0;
             const long long HW = (long long)g.H * g.W;
             const long long planes_total = (long long)g.N * g.C;
             const int KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP;
-            for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
-                const int ct_all = (int)(t % (g.ctiles * g.group));
+            for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
+                const int ct_all = (int)(t % cgt);
                 const int grp = ct_all / g.ctiles;
-                const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
-                // The segment table is the same for every channel block of the tile.  It lives beside
-                // the raw stage that carries the tile's first block and is written only once that stage
-                // has been released, so it cannot change under transform warps still working on an
-                // earlier tile; they read it after this stage has landed.
-                TcConvSegs *segs = nullptr;
-                int nseg = 0;
-                uint32_t tile_bytes = 0;
+                const long long G0 = ((t / cgt) * kCtas + rank) * tile_rows;
+                // The segment table is the same for every channel block of the tile.  Two tables
+                // alternate by tile; the transform warps hand a table back once they have turned it
+                // into their per-thread offsets, so it is ready long before the tile's data lands.
+                const uint32_t sp = tile_it & 1u;
+                mbar_wait(&bars->seg_empty[sp], ((tile_it >> 1) & 1u) ^ 1u, err, 20);
+                TcConvSegs *segs = reinterpret_cast<TcConvSegs *>(seg_st + sp * kSegBytes);
+                tc_conv_segments(g, G0, *segs);
+                mbar_arrive(&bars->seg_full[sp]);
+                ++tile_it;
+                const int nseg = segs->nseg;
+                const uint32_t tile_bytes = (uint32_t)segs->total_floats * 4u;
+                const int rot = cb_rotation(t, ncb);
                 for (int cb = 0; cb < ncb; ++cb) {
                     mbar_wait(&bars->raw_empty[rs], rphase ^ 1, err, 11);
-                    if (cb == 0) {
-                        segs = reinterpret_cast<TcConvSegs *>(seg_st + rs * kSegBytes);
-                        tc_conv_segments(g, G0, *segs);
-                        nseg = segs->nseg;
-                        tile_bytes = (uint32_t)segs->total_floats * 4u;
-                    }
+                    LOG(0, cb);
                     float *dst = reinterpret_cast<float *>(raw_st + (size_t)rs * g.raw_stage_bytes);
-                    const int c0 = grp * g.Cg + cb * KB;
+                    const int cbx = cb + rot < ncb ? cb + rot : cb + rot - ncb;
+                    const int c0 = grp * g.Cg + cbx * KB;
                     if (g.raw_mode == 0) {
                         mbar_arrive_expect_tx(&bars->raw_full[rs], tile_bytes);
                         for (int i = 0; i < nseg; ++i) {
@@ -217,8 +251,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                                              &bars->raw_full[rs]);
                         }
                     }
-                    rs ^= 1;
-                    if (rs == 0) rphase ^= 1;
+                    if (++rs == g.nr_stages) { rs = 0; rphase ^= 1; }
                 }
             }
         }
@@ -227,16 +260,20 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         if (elect_one()) {
             int bs = 0;
             uint32_t bphase = 0;
-            const long long per_ct = (long long)g.ncb * g.n_steps * g.b_step_bytes;   // bytes per channel tile
+            const long long per_ct = (long long)g.ncb * g.n_steps * g.b_step_bytes;   // bytes per channel tile and CTA
             const int nb = g.nb_stages, ncb = g.ncb, b_steps = g.b_steps, spb = g.spb, n_steps = g.n_steps;
             const uint32_t stage_bytes = (uint32_t)g.b_stage_bytes, step_bytes = (uint32_t)g.b_step_bytes;
-            for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
-                const int ct_all = (int)(t % (g.ctiles * g.group));
-                const uint8_t *src = reinterpret_cast<const uint8_t *>(Wpk) + ct_all * per_ct;
+            for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
+                const int ct_all = (int)(t % cgt);
+                const uint8_t *tile_src = reinterpret_cast<const uint8_t *>(Wpk) + (ct_all * kCtas + (int)rank) * per_ct;
+                const int rot = cb_rotation(t, ncb);
                 for (int cb = 0; cb < ncb; ++cb) {
+                    const int cbx = cb + rot < ncb ? cb + rot : cb + rot - ncb;
+                    const uint8_t *src = tile_src + (long long)cbx * n_steps * step_bytes;
                     for (int bstep = 0; bstep < b_steps; ++bstep) {
                         const uint32_t bytes = (uint32_t)min(spb, n_steps - bstep * spb) * step_bytes;
                         mbar_wait(&bars->b_empty[bs], bphase ^ 1, err, 12);
+                        LOG(1, cb * b_steps + bstep);
                         mbar_arrive_expect_tx(&bars->b_full[bs], bytes);
                         bulk_load_1d(b_st + (size_t)bs * stage_bytes, src, bytes, &bars->b_full[bs]);
                         src += bytes;
@@ -251,10 +288,26 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         // groups 128 bytes apart (SBO), the two 16-byte K chunks of one instruction LBO apart.  For
         // A the per-step table holds offset and LBO (a chunk pitch, or the distance between two taps);
         // all descriptor words are precomputed, a step costs a table read and a few adds.
-        if (elect_one()) {
+        if (kCtas == 2 && rank != 0) {
+            // Odd CTA of a pair: the even CTA issues the MMAs.  Tell it when each of this CTA's weight
+            // stages has landed (everything else reaches its barriers directly).
+            if (elect_one()) {
+                const uint32_t peer_b_full = map_to_cta(smem_u32(&bars->b_full[0]), 0);
+                const int ncb = g.ncb, nb = g.nb_stages, b_steps = g.b_steps;
+                int bs = 0;
+                uint32_t bphase = 0;
+                for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
+                    for (int i = 0; i < ncb * b_steps; ++i) {
+                        mbar_wait(&bars->b_full[bs], bphase, err, 19);
+                        mbar_arrive_remote(peer_b_full + (uint32_t)bs * 8u);
+                        if (++bs == nb) { bs = 0; bphase ^= 1; }
+                    }
+                }
+            }
+        } else if (elect_one()) {
             const uint32_t desc_hi = (128u >> 4) | (1u << 14);                 // SBO = 128, descriptor version 1
             const uint32_t a_base16 = (smem_u32(a_st) >> 4) & 0x3FFFu;
-            const uint32_t b_lo0 = ((smem_u32(b_st) >> 4) & 0x3FFFu) | (((uint32_t)g.BN * 16u >> 4) << 16);
+            const uint32_t b_lo0 = ((smem_u32(b_st) >> 4) & 0x3FFFu) | (((uint32_t)g.BNH * 16u >> 4) << 16);
             const uint32_t a_stage16 = (uint32_t)g.a_stage_bytes >> 4, b_stage16 = (uint32_t)g.b_stage_bytes >> 4;
             const uint32_t b_step16 = (uint32_t)g.b_step_bytes >> 4;
             const uint32_t idesc = g.idesc;
@@ -263,39 +316,61 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             int as = 0, bs = 0;
             uint32_t aphase = 0, bphase = 0, it = 0;
             PROF_DECL;
-            for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x, ++it) {
-                // accumulator buffer: two of them alternate when a tile needs only 256 TMEM columns
-                const uint32_t ab = two ? 0u : (it & 1u), use = two ? it : (it >> 1);
-                const uint32_t d0 = tmem_base + ab * 256u;
-                mbar_wait(&bars->acc_empty[ab], (use & 1u) ^ 1u, err, 13);
+            for (long long t = first_tile; t < g.total_tiles; t += tile_step, ++it) {
+                const uint32_t ab = acc_dbl ? (it & 1u) : 0u, use = acc_dbl ? (it >> 1) : it;
+                const uint32_t d0 = tmem_base + ab * 256u, d1 = d0 + mt_cols;
+                if (kCtas == 2) mbar_wait_cluster(&bars->acc_empty[ab], (use & 1u) ^ 1u, err, 13);
+                else mbar_wait(&bars->acc_empty[ab], (use & 1u) ^ 1u, err, 13);
                 tc_fence_after_sync();
                 PROF_MARK(0);
                 uint32_t accumulate = 0;
                 for (int cb = 0; cb < ncb; ++cb) {
-                    mbar_wait(&bars->a_full[as], aphase, err, 14);
+                    if (kCtas == 2) mbar_wait_cluster(&bars->a_full[as], aphase, err, 14);
+                    else mbar_wait(&bars->a_full[as], aphase, err, 14);
                     PROF_MARK(1);
+                    LOG(2, cb);
                     const uint32_t a_lo = a_base16 + (uint32_t)as * a_stage16;
                     for (int bstep = 0; bstep < b_steps; ++bstep) {
-                        mbar_wait(&bars->b_full[bs], bphase, err, 15);
+                        if (kCtas == 2) mbar_wait_cluster(&bars->b_full[bs], bphase, err, 15);
+                        else mbar_wait(&bars->b_full[bs], bphase, err, 15);
                         tc_fence_after_sync();
                         PROF_MARK(2);
-                        const int s0 = bstep * spb, s1 = min(n_steps, s0 + spb);
-                        uint32_t bl = b_lo0 + (uint32_t)bs * b_stage16;
-                        for (int s = s0; s < s1; ++s, bl += b_step16) {
-                            const uint32_t al = a_lo + g.step_a[s];
-                            mma_tf32_lohi(d0, al, desc_hi, bl, desc_hi, idesc, accumulate);
-                            if (two) mma_tf32_lohi(d0 + 256u, al + 128u, desc_hi, bl, desc_hi, idesc, accumulate);
-                            accumulate = 1;
+                        LOG(3, cb * b_steps + bstep);
+                        // One thread issues everything, so every dependent instruction here costs
+                        // its full latency: fetch the stage's table entries together, then issue
+                        // the MMAs back to back with nothing but adds in between.
+                        const int s0 = bstep * spb, cnt = min(n_steps - s0, spb);
+                        const uint32_t bl = b_lo0 + (uint32_t)bs * b_stage16;
+                        uint32_t sa[kMaxSpb];
+#pragma unroll
+                        for (int j = 0; j < kMaxSpb; ++j) sa[j] = j < cnt ? g.step_a[s0 + j] : 0u;
+#pragma unroll
+                        for (int j = 0; j < kMaxSpb; ++j) {
+                            if (j < cnt) {
+                                const uint32_t al = a_lo + sa[j], blj = bl + (uint32_t)j * b_step16;
+                                if (kCtas == 2) {
+                                    mma_tf32_lohi_pair(d0, al, desc_hi, blj, desc_hi, idesc, accumulate);
+                                    if (two) mma_tf32_lohi_pair(d1, al + 128u, desc_hi, blj, desc_hi, idesc, accumulate);
+                                } else {
+                                    mma_tf32_lohi(d0, al, desc_hi, blj, desc_hi, idesc, accumulate);
+                                    if (two) mma_tf32_lohi(d1, al + 128u, desc_hi, blj, desc_hi, idesc, accumulate);
+                                }
+                                accumulate = 1;
+                            }
                         }
-                        mma_commit(&bars->b_empty[bs]);
+                        if (kCtas == 2) mma_commit_pair(&bars->b_empty[bs]);
+                        else mma_commit(&bars->b_empty[bs]);
                         if (++bs == nb) { bs = 0; bphase ^= 1; }
                         PROF_MARK(3);
                     }
-                    mma_commit(&bars->a_empty[as]);
+                    if (kCtas == 2) mma_commit_pair(&bars->a_empty[as]);
+                    else mma_commit(&bars->a_empty[as]);
+                    LOG(4, cb);
                     as ^= 1;
                     if (as == 0) aphase ^= 1;
                 }
-                mma_commit(&bars->acc_full[ab]);
+                if (kCtas == 2) mma_commit_pair(&bars->acc_full[ab]);
+                else mma_commit(&bars->acc_full[ab]);
                 PROF_MARK(4);
             }
             PROF_FLUSH(0);
@@ -306,66 +381,106 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         const int xt = xw * 32 + lane;             // 0..255
         const int cp = g.raw_mode == 1 ? g.H * g.W : g.BOXP;    // channel pitch inside the raw stage
         const int per_stage_slots = g.planes * g.SLOTS;
-        const int nchunks = g.nchunks, KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP;
-        const uint32_t chunk_pitch = (uint32_t)g.chunk_pitch;
+        const int nchunks = g.nchunks, KB = g.KB, ncb = g.ncb, box_floats = g.KB * g.BOXP, nr = g.nr_stages;
+        // Work units: one (slot, 4-channel chunk) pair = four raw reads and one 16-byte operand row.
+        // Unit u = chunk * slots + slot; this thread owns units xt, xt + 256, ...
+        const int units = per_stage_slots * nchunks;
+        const int nu = (units - xt + kXformThreads - 1) / kXformThreads;
         int rs = 0, as = 0;
-        uint32_t rphase = 0, aphase = 0;
+        uint32_t rphase = 0, aphase = 0, tile_it = 0;
         PROF_DECL;
-        for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x) {
-            const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
-            int off[kOwned];                       // raw float offset of channel 0 for the slots this thread owns
-            for (int cb = 0; cb < ncb; ++cb) {
-                mbar_wait(&bars->raw_full[rs], rphase, err, 16);
-                PROF_MARK(0);
-                if (cb == 0) {
-                    const TcConvSegs *segs = reinterpret_cast<const TcConvSegs *>(seg_st + rs * kSegBytes);
+        const uint32_t a_full_addr = kCtas == 2 ? map_to_cta(smem_u32(&bars->a_full[0]), 0) : 0u;
+        for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
+            const long long G0 = ((t / cgt) * kCtas + rank) * tile_rows;
+            int uoff[kOwned];                      // raw float offset of the unit's first channel, -1 = padding
+            uint32_t udst[kOwned];                 // byte offset of the unit's operand row inside an A stage
+            const int rot = cb_rotation(t, ncb);
+            {
+                // per-thread offsets of the tile, from its segment table (ready before the data)
+                const uint32_t sp = tile_it & 1u;
+                mbar_wait(&bars->seg_full[sp], (tile_it >> 1) & 1u, err, 21);
+                ++tile_it;
+                const TcConvSegs *segs = reinterpret_cast<const TcConvSegs *>(seg_st + sp * kSegBytes);
 #pragma unroll
-                    for (int i = 0; i < kOwned; ++i) {
-                        off[i] = -1;
-                        const int idx = xt + i * kXformThreads;
-                        if (idx < per_stage_slots) {
-                            const int pl = idx / g.SLOTS, j = idx - pl * g.SLOTS;
-                            const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
-                            if (Gs < (uint32_t)g.total_slots) {
-                                const int n = (int)(Gs / (uint32_t)g.L);
-                                const int u = (int)(Gs - (uint32_t)n * (uint32_t)g.L);
-                                const int hq = u / g.Ws, wq = u - hq * g.Ws;
-                                const int h = hq * g.sh + g.pa[pl] - g.pt;
-                                const int w = wq * g.sw + g.pb[pl] - g.pl;
-                                const int sg = n - segs->n_first;
-                                if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
-                                    const int f = h * g.W + w - segs->f0[sg];
-                                    if (g.raw_mode == 1) off[i] = segs->base[sg] + f;
-                                    else {
-                                        const int bx = f / g.BOXP;
-                                        off[i] = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
-                                    }
+                for (int i = 0; i < kOwned; ++i) {
+                    uoff[i] = -1;
+                    udst[i] = 0;
+                    if (i < nu) {
+                        const int u = xt + i * kXformThreads;
+                        const int ch = conv_fdiv(u, per_stage_slots, g.inv_pss), idx = u - ch * per_stage_slots;
+                        udst[i] = (uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u;
+                        const int pl = conv_fdiv(idx, g.SLOTS, g.inv_SLOTS), j = idx - pl * g.SLOTS;
+                        const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
+                        if (Gs < (uint32_t)g.total_slots) {
+                            const int n = conv_fdiv((int)Gs, g.L, g.inv_L);
+                            const int uu = (int)Gs - n * g.L;
+                            const int hq = conv_fdiv(uu, g.Ws, g.inv_Ws), wq = uu - hq * g.Ws;
+                            const int h = hq * g.sh + g.pa[pl] - g.pt;
+                            const int w = wq * g.sw + g.pb[pl] - g.pl;
+                            const int sg = n - segs->n_first;
+                            if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
+                                const int f = h * g.W + w - segs->f0[sg];
+                                int o;
+                                if (g.raw_mode == 1) o = segs->base[sg] + f;
+                                else {
+                                    const int bx = conv_fdiv(f, g.BOXP, g.inv_BOXP);
+                                    o = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
                                 }
+                                uoff[i] = o + ch * 4 * cp;
                             }
                         }
                     }
-                    PROF_MARK(2);
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->seg_empty[sp]);
+                PROF_MARK(2);
+            }
+            for (int cb = 0; cb < ncb; ++cb) {
+                mbar_wait(&bars->raw_full[rs], rphase, err, 16);
+                PROF_MARK(0);
+                if (xt == 0) LOG(5, cb);
                 mbar_wait(&bars->a_empty[as], aphase ^ 1, err, 17);
                 PROF_MARK(1);
+                if (xt == 0) LOG(6, cb);
                 const float *raw = reinterpret_cast<const float *>(raw_st + (size_t)rs * g.raw_stage_bytes);
                 uint8_t *adst = a_st + (size_t)as * g.a_stage_bytes;
-                const int c_left = g.Cg - cb * KB;     // channels of this block that exist
+                const int cbx = cb + rot < ncb ? cb + rot : cb + rot - ncb;
+                const int c_left = g.Cg - cbx * KB;    // channels of this block that exist
+                if (c_left >= KB) {
+                    // every channel of the block exists: all reads first, then round and store
+                    float v[kOwned][4];
 #pragma unroll
-                for (int i = 0; i < kOwned; ++i) {
-                    const int idx = xt + i * kXformThreads;
-                    if (idx < per_stage_slots) {
-                        for (int ch = 0; ch < nchunks; ++ch) {
+                    for (int i = 0; i < kOwned; ++i) {
+                        v[i][0] = v[i][1] = v[i][2] = v[i][3] = 0.f;
+                        if (i < nu && uoff[i] >= 0) {
+                            const float *r = raw + uoff[i];
+                            v[i][0] = r[0];
+                            v[i][1] = r[cp];
+                            v[i][2] = r[2 * cp];
+                            v[i][3] = r[3 * cp];
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < kOwned; ++i)
+                        if (i < nu)
+                            *reinterpret_cast<float4 *>(adst + udst[i]) =
+                                make_float4(round_tf32(v[i][0]), round_tf32(v[i][1]), round_tf32(v[i][2]),
+                                            round_tf32(v[i][3]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kOwned; ++i) {
+                        if (i < nu) {
                             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (off[i] >= 0) {
-                                const float *r = raw + off[i] + (ch * 4) * cp;
+                            if (uoff[i] >= 0) {
+                                const float *r = raw + uoff[i];
+                                const int ch = (xt + i * kXformThreads) / per_stage_slots;
                                 const int left = c_left - ch * 4;
                                 if (left > 0) v.x = round_tf32(r[0]);
                                 if (left > 1) v.y = round_tf32(r[cp]);
                                 if (left > 2) v.z = round_tf32(r[2 * cp]);
                                 if (left > 3) v.w = round_tf32(r[3 * cp]);
                             }
-                            *reinterpret_cast<float4 *>(adst + (size_t)ch * chunk_pitch + (size_t)idx * 16) = v;
+                            *reinterpret_cast<float4 *>(adst + udst[i]) = v;
                         }
                     }
                 }
@@ -373,12 +488,13 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(&bars->a_full[as]);
+                    if (kCtas == 2) mbar_arrive_remote(a_full_addr + (uint32_t)as * 8u);   // the issuing CTA's barrier
+                    else mbar_arrive(&bars->a_full[as]);
                     mbar_arrive(&bars->raw_empty[rs]);
                 }
                 PROF_MARK(3);
-                rs ^= 1;
-                if (rs == 0) rphase ^= 1;
+                if (xt == 0) LOG(7, cb);
+                if (++rs == nr) { rs = 0; rphase ^= 1; }
                 as ^= 1;
                 if (as == 0) aphase ^= 1;
             }
@@ -392,19 +508,20 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         const int hf = ew >> 2;
         const long long PQ = (long long)g.P * g.Q;
         const bool two = g.MT == 2;
+        const uint32_t acc_empty_addr = kCtas == 2 ? map_to_cta(smem_u32(&bars->acc_empty[0]), 0) : 0u;
         uint32_t it = 0;
-        for (long long t = blockIdx.x; t < g.total_tiles; t += gridDim.x, ++it) {
-            const int ct_all = (int)(t % (g.ctiles * g.group));
+        for (long long t = first_tile; t < g.total_tiles; t += tile_step, ++it) {
+            const int ct_all = (int)(t % cgt);
             const int grp = ct_all / g.ctiles, ct = ct_all % g.ctiles;
-            const long long G0 = (t / (g.ctiles * g.group)) * tile_rows;
-            const uint32_t ab = two ? 0u : (it & 1u), use = two ? it : (it >> 1);
+            const long long G0 = ((t / cgt) * kCtas + rank) * tile_rows;
+            const uint32_t ab = acc_dbl ? (it & 1u) : 0u, use = acc_dbl ? (it >> 1) : it;
             mbar_wait(&bars->acc_full[ab], use & 1u, err, 18);
             tc_fence_after_sync();
             const int nch = (g.BN + 31) / 32;
             int mt, ch_lo, ch_hi;
             if (two) { mt = hf; ch_lo = 0; ch_hi = nch; }
             else { mt = 0; ch_lo = hf ? (nch + 1) / 2 : 0; ch_hi = hf ? nch : (nch + 1) / 2; }
-            const uint32_t acc_col = two ? (uint32_t)mt * 256u : ab * 256u;
+            const uint32_t acc_col = ab * 256u + (uint32_t)mt * mt_cols;
             const uint32_t G = (uint32_t)G0 + (uint32_t)(mt * 128 + quarter * 32 + lane);
             bool valid = G < (uint32_t)g.total_slots;
             float *yrow = Y;
@@ -434,12 +551,16 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);
+            if (lane == 0) {
+                if (kCtas == 2) mbar_arrive_remote(acc_empty_addr + ab * 8u);
+                else mbar_arrive(&bars->acc_empty[ab]);
+            }
         }
     }
 
     tc_fence_before_sync();
     __syncthreads();
+    if (kCtas == 2) cluster_sync_all();     // no CTA leaves while its peer may still signal it
     if (warp == 2) {
         __syncwarp();
         tc_fence_after_sync();
@@ -492,7 +613,10 @@ int pick_conv_bn(int Mg) {
     return best;
 }
 
-bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
+bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, TcConvPlan &g) {
+    if (ctas == 2 && BN % 16) return false;      // M = 256 instructions take N in multiples of 16
+    g.ctas = ctas;
+    g.BNH = BN / ctas;
     g.N = c.N; g.C = c.C; g.H = c.H; g.W = c.W; g.M = c.M; g.Cg = c.Cg; g.Mg = c.Mg;
     g.kH = c.kH; g.kW = c.kW; g.P = c.P; g.Q = c.Q; g.pt = c.pt; g.pl = c.pl;
     g.sh = c.sh; g.sw = c.sw; g.dh = c.dh; g.dw = c.dw; g.group = c.group; g.relu = c.relu;
@@ -516,7 +640,7 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     g.MT = MT; g.BN = BN;
     g.ctiles = (c.Mg + BN - 1) / BN;
     const long long slots = (long long)MT * 128 + maxshift;
-    if (slots * g.planes > kOwned * kXformThreads) return false;
+    if (slots * g.planes * (c.Cg >= 16 ? 4 : 1) > kOwned * kXformThreads) return false;
     g.SLOTS = (int)slots;
     if ((g.SLOTS + L - 2) / L + 1 > kConvMaxSeg) return false;
     g.plane_pitch = g.SLOTS * 16;
@@ -577,10 +701,10 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     }
     g.nchunks = g.KB / 4;
     g.ncb = (c.Cg + g.KB - 1) / g.KB;
-    const long long ptiles = (g.total_slots + MT * 128 - 1) / (MT * 128);
+    const long long ptiles = (g.total_slots + MT * 128 - 1) / (MT * 128);      // per-CTA pixel tiles
     if (ptiles > 0x7fffffffLL) return false;
-    g.pix_tiles = (int)ptiles;
-    g.total_tiles = ptiles * g.ctiles * c.group;
+    g.pix_tiles = (int)((ptiles + ctas - 1) / ctas);
+    g.total_tiles = (long long)g.pix_tiles * g.ctiles * c.group;
     // raw staging mode
     const long long HW = (long long)c.H * c.W;
     if (HW % 4 == 0) {
@@ -592,10 +716,10 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
     }
     g.a_stage_bytes = g.nchunks * g.chunk_pitch;
     g.a_stage_bytes = (g.a_stage_bytes + 127) / 128 * 128;
-    g.b_step_bytes = BN * 32;
-    g.spb = std::max(1, std::min(g.n_steps, 32768 / g.b_step_bytes));   // several K-steps per weight stage
-    g.idesc = tc::make_idesc_tf32(128, BN, 0, 0);
-    g.packed_floats = (long long)c.group * g.ctiles * g.ncb * g.n_steps * BN * 8;
+    g.b_step_bytes = g.BNH * 32;
+    g.spb = std::max(1, std::min(std::min(g.n_steps, kMaxSpb), 32768 / g.b_step_bytes));   // several K-steps per weight stage
+    g.idesc = tc::make_idesc_tf32(128 * ctas, BN, 0, 0);
+    g.packed_floats = (long long)c.group * g.ctiles * g.ncb * g.n_steps * BN * 8;     // both CTAs' parts
     // raw stage size: widest flat pixel range any tile needs, found by walking the tiles
     g.BOXP = 256;
     const long long walk = std::min<long long>(ptiles, L + 2);
@@ -634,13 +758,24 @@ bool fill_plan(const ConvGeom &c, int MT, int BN, TcConvPlan &g) {
         g.raw_stage_bytes = (worst * 4 + 127) / 128 * 128;
         if (g.raw_stage_bytes == 0) g.raw_stage_bytes = 128;
     }
-    const long long fixed = 1024 + 2LL * g.a_stage_bytes + 2LL * g.raw_stage_bytes + 2 * kSegBytes + kBarBytes;
+    // Raw stages: a third one (the raw tiles come from L2/HBM with a microsecond of latency) when that
+    // still leaves 64 KB for the weight ring.
+    const long long base_fixed = 1024 + 2LL * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
+    g.nr_stages = 2;
+    for (int nr = 3; nr <= kMaxRawStages - 1; ++nr)
+        if (kSmemLimit - base_fixed - (long long)nr * g.raw_stage_bytes >= 65536) g.nr_stages = nr;
+    const long long fixed = base_fixed + (long long)g.nr_stages * g.raw_stage_bytes;
     const long long room = kSmemLimit - fixed;
     while (room < 3LL * g.spb * g.b_step_bytes && g.spb > 1) g.spb = (g.spb + 1) / 2;   // keep three stages in flight
     g.b_steps = (g.n_steps + g.spb - 1) / g.spb;
     g.b_stage_bytes = g.spb * g.b_step_bytes;
     if (room < 2LL * g.b_stage_bytes) return false;
     g.nb_stages = (int)std::min<long long>(kMaxBStages, room / g.b_stage_bytes);
+    g.inv_L = conv_recip(g.L);
+    g.inv_Ws = conv_recip(g.Ws);
+    g.inv_BOXP = conv_recip(g.BOXP);
+    g.inv_SLOTS = conv_recip(g.SLOTS);
+    g.inv_pss = conv_recip(g.planes * g.SLOTS);
     return true;
 }
 
@@ -656,32 +791,56 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
     }
     const int sms = 148;
     const int bn0 = pick_conv_bn(c.Mg);
-    int cand[5][2];
+    // candidate tiles (CTAs per tile, accumulators per CTA, channels per tile)
+    int cand[16][3];
     int ncand = 0;
-    cand[ncand][0] = 2; cand[ncand++][1] = bn0;
-    cand[ncand][0] = 1; cand[ncand++][1] = bn0;
-    if (bn0 > 128) {
-        cand[ncand][0] = 2; cand[ncand++][1] = 128;
-        cand[ncand][0] = 1; cand[ncand++][1] = 128;
+    auto add = [&](int ctas, int mt, int bn) {
+        for (int i = 0; i < ncand; ++i)
+            if (cand[i][0] == ctas && cand[i][1] == mt && cand[i][2] == bn) return;
+        cand[ncand][0] = ctas; cand[ncand][1] = mt; cand[ncand][2] = bn; ++ncand;
+    };
+    int fc = 0, fm = 0, fb = 0;
+    if (const char *e = getenv("ONNXB_CONV_TILE")) {      // "ctas,MT,BN": pin the tile for A/B measurements
+        if (sscanf(e, "%d,%d,%d", &fc, &fm, &fb) == 3 && (fc == 1 || fc == 2) && (fm == 1 || fm == 2) && fb >= 16 &&
+            fb <= 256 && fb % 16 == 0)
+            add(fc, fm, fb);
     }
-    if (bn0 > 64) { cand[ncand][0] = 1; cand[ncand++][1] = 64; }
+    if (ncand == 0) {
+        for (int ctas = 2; ctas >= 1; --ctas) {
+            add(ctas, 2, bn0);
+            add(ctas, 1, bn0);
+            if (bn0 > 128) { add(ctas, 2, 128); add(ctas, 1, 128); }
+            if (bn0 > 64) add(ctas, 1, 64);
+        }
+    }
     bool have = false;
     double best_cost = 0;
     for (int i = 0; i < ncand; ++i) {
         TcConvPlan p;
-        if (!fill_plan(c, cand[i][0], cand[i][1], p)) continue;
-        // Cost in SM cycles.  Per channel block the slowest of: the transform warps (about 200 + 420
-        // cycles per 256 slots and chunk quartet), the tensor pipe (BN/2 cycles per instruction, or the
-        // shared-memory time of its operands when that is longer) and the weight stream out of L2
-        // (about 3600 bytes per cycle over all SMs, at most 64 per SM).
-        const long long waves = (p.total_tiles + sms - 1) / sms;
-        const double active = (double)std::min<long long>(p.total_tiles, sms);
-        const double t_x = (200.0 + 420.0 * ((p.planes * p.SLOTS + 255) / 256)) * p.nchunks / 4.0;
-        const double t_inst = std::max(p.BN / 2.0, 40.0 + p.BN / 4.0) * (p.BN <= 128 ? 1.25 : 1.0);
-        const double t_mma = (double)p.n_steps * p.MT * t_inst;
-        const double t_w = (double)p.n_steps * p.b_step_bytes / std::min(64.0, 3600.0 / active);
-        const double per_cb = std::max(t_x, std::max(t_mma, t_w));
-        const double cost = (double)waves * (p.ncb * per_cb + 3000.0 + 8.0 * p.MT * p.BN);
+        if (!fill_plan(c, cand[i][0], cand[i][1], cand[i][2], p)) continue;
+        // Cost in SM cycles per CTA, fitted to measured tile sweeps of the ResNet-50 3x3 layers.  Per
+        // channel block the slowest of: the tensor pipe (BN/2 cycles per 128 x BN x 8 share of an
+        // instruction, or the 128 bytes/cycle of shared memory its operands need, whichever is longer),
+        // shared memory as a whole (operand reads plus the stages written and the transform, at about
+        // 90 bytes/cycle sustained), the weight stream out of L2 (about 3600 bytes/cycle over all SMs, at
+        // most 48 per SM) and the transform warps; plus a fixed hand-over cost per block, larger for
+        // pairs (their barriers cross the cluster).
+        const int units = sms / p.ctas;                                     // tiles in flight
+        const long long waves = (p.total_tiles + units - 1) / units;
+        const double active = (double)std::min<long long>(p.total_tiles, units) * p.ctas;
+        const double n_inst = (double)p.n_steps * p.MT;
+        const double op_bytes = 4096.0 + p.BNH * 32.0;
+        const double t_mma = n_inst * (std::max(p.BN / 2.0, op_bytes / 128.0) + (p.ctas == 2 ? 10.0 : 0.0));
+        const double w_bytes = (double)p.n_steps * p.b_step_bytes;
+        const double slots16 = (double)p.planes * p.SLOTS * 16.0 * p.nchunks;
+        const double t_smem = (n_inst * op_bytes + w_bytes + 3.0 * slots16) / 90.0;
+        const double t_w = w_bytes / std::min(48.0, 3600.0 / active);
+        const double t_x = 300.0 + 100.0 * ((p.planes * p.SLOTS * p.nchunks + 255) / 256);
+        const double per_cb = std::max(std::max(t_mma, t_smem), std::max(t_w, t_x)) + 400.0 + (p.ctas == 2 ? 700.0 : 0.0);
+        const bool dbl = p.MT == 1 || p.BN <= 128;
+        const double t_epi = 8.0 * p.MT * p.BN;                             // read-back and stores of one tile
+        const double per_tile = (dbl ? std::max(p.ncb * per_cb, t_epi) : p.ncb * per_cb + t_epi) + 3000.0;
+        const double cost = (double)waves * per_tile + 9000.0 + (dbl ? t_epi : 0.0);
         if (!have || cost < best_cost * 0.999) {
             have = true;
             best_cost = cost;
@@ -702,9 +861,41 @@ extern "C" int onnxb_dbg_check(long long *out) {
 extern "C" int onnxb_dbg_profile(long long *out) {
     cudaDeviceSynchronize();
     cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 148 * 16);
+    static long long zeros[148 * 16];
+    cudaMemcpyToSymbol(g_prof, zeros, sizeof zeros);
+    return 0;
+}
+extern "C" int onnxb_dbg_log(long long *out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_log, sizeof(long long) * 8 * 64);
     return 0;
 }
 #endif
+
+// How many CTA pairs (clusters of two) of the pair kernel the device runs at once; queried once.
+static int max_pairs(size_t smem) {
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * 148);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemLimit;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    (void)smem;
+    if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2>, &cfg) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = tc_host::num_sms() / 2;
+    }
+    cached = n;
+    return n;
+}
 
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan) { return (size_t)plan.packed_floats * 4; }
 
@@ -734,20 +925,28 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     } else {
         memset(&tmX, 0, sizeof tmX);
     }
-    const size_t smem = 1024 + 2 * (size_t)plan.a_stage_bytes + 2 * (size_t)plan.raw_stage_bytes +
-                        (size_t)plan.nb_stages * plan.b_stage_bytes + 2 * kSegBytes + kBarBytes;
-    cudaError_t e = cudaFuncSetAttribute(tc_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    const size_t smem = 1024 + 2 * (size_t)plan.a_stage_bytes + (size_t)plan.nr_stages * plan.raw_stage_bytes +
+                        (size_t)plan.nb_stages * plan.b_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
+    const bool pair = plan.ctas == 2;
+    cudaError_t e = cudaFuncSetAttribute(pair ? tc_conv_kernel<2> : tc_conv_kernel<1>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return (int)e;
     const int sms = num_sms();
-    const int grid = (int)std::min<long long>(plan.total_tiles, sms);
+    // persistent: one CTA per SM; pairs are clusters of two neighbouring SMs
+    const int units = pair ? max_pairs(smem) : sms;
+    if (units < 1) return (int)cudaErrorLaunchOutOfResources;
+    const int grid = (int)std::min<long long>(plan.total_tiles, units) * plan.ctas;
 #ifdef ONNXB_PROFILE
-    fprintf(stderr, "[plan] MT %d BN %d ctiles %d SLOTS %d planes %d Hs %d Ws %d L %d KB %d ncb %d steps %d spb %d tiles %lld grid %d raw_mode %d BOXP %d a_stage %d raw_stage %d b_stage %d nb %d smem %zu\n",
-            plan.MT, plan.BN, plan.ctiles, plan.SLOTS, plan.planes, plan.Hs, plan.Ws, plan.L, plan.KB, plan.ncb,
+    fprintf(stderr, "[plan] ctas %d MT %d BN %d ctiles %d SLOTS %d planes %d Hs %d Ws %d L %d KB %d ncb %d steps %d spb %d tiles %lld grid %d raw_mode %d BOXP %d a_stage %d raw_stage %d b_stage %d nb %d smem %zu\n",
+            plan.ctas, plan.MT, plan.BN, plan.ctiles, plan.SLOTS, plan.planes, plan.Hs, plan.Ws, plan.L, plan.KB, plan.ncb,
             plan.n_steps, plan.spb, plan.total_tiles, grid, plan.raw_mode, plan.BOXP, plan.a_stage_bytes,
             plan.raw_stage_bytes, plan.b_stage_bytes, plan.nb_stages, smem);
 #endif
-    const cudaError_t le = launch_pdl(tc_conv_kernel, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
-                                      reinterpret_cast<const float *>(workspace), B, Y, err);
+    const cudaError_t le =
+        pair ? launch_pdl_cluster(tc_conv_kernel<2>, 2, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+                                  reinterpret_cast<const float *>(workspace), B, Y, err)
+             : launch_pdl(tc_conv_kernel<1>, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+                          reinterpret_cast<const float *>(workspace), B, Y, err);
     count_launch();
     return (int)le;
 }

@@ -44,22 +44,40 @@ struct TcConvPlan {
     short src_tap[kConvMaxSteps][2];     // which filter tap feeds chunk 0 / 1 of the step's weights (-1: zeros)
     short src_c0[kConvMaxSteps][2];      // and from which channel offset inside the block
     // tiling
-    int MT;                          // 128-row accumulator tiles per CTA tile (1 or 2)
+    int ctas;                        // CTAs working on one tile: 1, or 2 (a cluster pair issuing M = 256 MMAs)
+    int MT;                          // 128-row accumulator tiles per CTA (1 or 2)
     int BN, ctiles;                  // output channels per tile, tiles per group
+    int BNH;                         // weight rows each CTA stages per K-step = BN / ctas
     int SLOTS;                       // slots per plane held in one A stage = MT*128 + largest tap shift
     int ncb;                         // channel blocks = ceil(Cg / KB)
-    int pix_tiles;                   // ceil(total_slots / (MT*128))
+    int pix_tiles;                   // ceil(total_slots / (ctas*MT*128))
     long long total_tiles;
     // raw staging
     int raw_mode;                    // 0: tensor-map boxes [KB][BOXP] over X seen as (H*W, N*C); 1: whole-image slabs
     int BOXP;
     // shared memory carve-up (bytes)
-    int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages;
+    int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages, nr_stages;
     int spb, b_step_bytes, b_steps;  // K-steps per weight stage, bytes of one step's weights, weight stages per block
     int chunk_pitch, plane_pitch;    // bytes between 4-channel chunks / parity planes inside an A stage
     uint32_t idesc;
     long long packed_floats;         // size of the packed weight buffer
+    // reciprocals (nudged up by 2^-40) of the divisors device code needs per slot: see conv_fdiv
+    double inv_L, inv_Ws, inv_BOXP, inv_SLOTS, inv_pss;
 };
+
+// floor(n / d) for 0 <= n < 2^31.  On the device: one double multiply by the stored reciprocal
+// (exact: the nudge keeps the product at or above the true quotient and the overshoot stays below
+// 1/d); on the host: plain integer division.
+ONNXB_HD inline int conv_fdiv(int n, int d, double inv) {
+#if defined(__CUDA_ARCH__)
+    (void)d;
+    return __double2int_rd((double)n * inv);
+#else
+    (void)inv;
+    return n / d;
+#endif
+}
+inline double conv_recip(int d) { return (1.0 / (double)d) * (1.0 + 1.0 / 1099511627776.0); }
 
 struct TcConvSegs {
     int n_first, nseg;
@@ -73,8 +91,14 @@ struct TcConvSegs {
 ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvSegs &t) {
     long long Gend = G0 + g.SLOTS;
     if (Gend > g.total_slots) Gend = g.total_slots;
-    t.n_first = (int)(G0 / g.L);
-    const int n_last = (int)((Gend - 1) / g.L);
+    if (G0 >= g.total_slots) {       // the second CTA of a pair on the last, half-empty tile
+        t.n_first = g.N;
+        t.nseg = 0;
+        t.total_floats = 0;
+        return;
+    }
+    t.n_first = conv_fdiv((int)G0, g.L, g.inv_L);
+    const int n_last = conv_fdiv((int)(Gend - 1), g.L, g.inv_L);
     t.nseg = n_last - t.n_first + 1;
     if (t.nseg > kConvMaxSeg) t.nseg = kConvMaxSeg;   // excluded by the planner
     int base = 0;
@@ -83,7 +107,7 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
         const long long lo = G0 > n * g.L ? G0 : n * g.L;
         const long long hi = Gend < (n + 1) * g.L ? Gend : (n + 1) * g.L;
         const int u_lo = (int)(lo - n * g.L), u_hi = (int)(hi - n * g.L);   // [u_lo, u_hi)
-        const int hq_lo = u_lo / g.Ws, hq_hi = (u_hi - 1) / g.Ws;
+        const int hq_lo = conv_fdiv(u_lo, g.Ws, g.inv_Ws), hq_hi = conv_fdiv(u_hi - 1, g.Ws, g.inv_Ws);
         int h_min = hq_lo * g.sh + g.a_min - g.pt;
         int h_max = hq_hi * g.sh + g.a_max - g.pt;
         if (h_min < 0) h_min = 0;
@@ -100,7 +124,7 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
             const int f0 = (h_min * g.W) & ~3;
             const int len = (h_max + 1) * g.W - f0;
             t.f0[i] = f0;
-            t.nbox[i] = (len + g.BOXP - 1) / g.BOXP;
+            t.nbox[i] = conv_fdiv(len + g.BOXP - 1, g.BOXP, g.inv_BOXP);
             base += t.nbox[i] * g.BOXP * g.KB;
         }
     }

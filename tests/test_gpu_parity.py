@@ -151,6 +151,37 @@ def test_conv_forced_implicit_gemm(binding, c):
     assert worst_ratio(got, want, S) <= 1.0
 
 
+# every tile shape of the implicit-GEMM kernel, single CTA and CTA pair (cluster of two, M = 256
+# instructions), on shapes with several tiles, a half-empty last pair tile, groups and ragged channels
+TILE_CASES = [
+    dict(x=(3, 32, 30, 30), w=(64, 32, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(5, 48, 14, 14), w=(272, 48, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(2, 64, 20, 20), w=(96, 16, 3, 3), pads=(1, 1, 1, 1), group=4),
+    dict(x=(9, 32, 7, 7), w=(144, 32, 3, 3), pads=(1, 1, 1, 1)),
+    dict(x=(2, 3, 64, 64), w=(64, 3, 7, 7), pads=(3, 3, 3, 3), strides=(2, 2)),
+]
+
+
+@pytest.mark.parametrize("tile", ["1,1,64", "1,2,64", "1,2,128", "1,1,256", "2,1,64", "2,2,64", "2,2,128", "2,1,256",
+                                  "2,2,256", "2,1,48"])
+@pytest.mark.parametrize("c", TILE_CASES, ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+def test_conv_implicit_gemm_tile_shapes(binding, c, tile, monkeypatch):
+    rng = np.random.default_rng(99)
+    X = rng.standard_normal(c["x"]).astype(np.float32)
+    W = rng.standard_normal(c["w"]).astype(np.float32)
+    B = rng.standard_normal((c["w"][0],)).astype(np.float32)
+    kw = dict(pads=c.get("pads", (0, 0, 0, 0)), strides=c.get("strides", (1, 1)), group=c.get("group", 1))
+    monkeypatch.setenv("ONNXB_CONV_TILE", tile)      # read when the descriptor is created
+    binding.set_kernel_override("mma_implicit")
+    try:
+        got, fam = run_conv_gpu(binding, torch, X, W, B, relu=False, **kw)
+    finally:
+        binding.set_kernel_override(None)
+    assert fam == "mma_implicit"
+    want, S = oracle.conv2d(X, W, B, relu=False, **kw)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 def test_conv_auto_pad_and_no_bias(binding):
     rng = np.random.default_rng(5)
     X = rng.standard_normal((2, 6, 13, 11)).astype(np.float32)
