@@ -213,6 +213,120 @@ gather1x1_vec_kernel(const float4 *__restrict__ X4, float4 *__restrict__ Xg4, un
     }
 }
 
+// Depthwise convolution with unit stride and dilation (group = C = M), the HBM-bound case: 2.25
+// flop per byte, so the only thing that matters is to move each plane once with few instructions.
+// A thread owns a strip of 4 output columns by 2 output rows of one (image, channel) plane, reads
+// the KH + 1 input rows it needs straight from global memory (neighbouring threads' overlapping
+// reads are served by L1) and keeps the window in registers: 21 loads and 72 FMAs for 8 outputs of
+// a 3x3 filter.  VEC: the row pitch and the left pad allow one aligned 16-byte load per row for the
+// strip's middle columns; otherwise every column is loaded on its own.
+template <int KH, int KW, bool VEC>
+__global__ void __launch_bounds__(256)
+conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
+                             const float *__restrict__ B, float *__restrict__ Y, unsigned items, unsigned Q4,
+                             unsigned P2, double inv_Q4, double inv_P2) {
+    constexpr int WIN = KW + 3;                // input columns a strip of 4 outputs touches
+    const unsigned i = blockIdx.x * 256u + threadIdx.x;
+    if (i >= items) return;
+    // i = (plane * P2 + row pair) * Q4 + column quad; quotients by reciprocal multiplication in
+    // double (right for 31-bit operands up to one unit, which the two comparisons repair)
+    unsigned t = __double2uint_rd((double)i * inv_Q4);
+    if (t * Q4 > i) --t;
+    if ((t + 1) * Q4 <= i) ++t;
+    const unsigned q4 = i - t * Q4;
+    unsigned plane = __double2uint_rd((double)t * inv_P2);
+    if (plane * P2 > t) --plane;
+    if ((plane + 1) * P2 <= t) ++plane;
+    const int p0 = (int)(t - plane * P2) * 2, q0 = (int)q4 * 4;
+    const int c = (int)(plane % (unsigned)g.C);
+
+    float w[KH * KW];
+#pragma unroll
+    for (int k = 0; k < KH * KW; ++k) w[k] = __ldg(W + (size_t)c * (KH * KW) + k);
+    const float bias = B ? __ldg(B + c) : 0.f;
+    float acc0[4] = {bias, bias, bias, bias}, acc1[4] = {bias, bias, bias, bias};
+
+    const float *xp = X + (size_t)plane * g.H * g.W;
+    const int iw0 = q0 - g.pl;
+#pragma unroll
+    for (int rr = 0; rr < KH + 1; ++rr) {
+        const int ih = p0 - g.pt + rr;
+        float v[WIN];
+#pragma unroll
+        for (int k = 0; k < WIN; ++k) v[k] = 0.f;
+        if ((unsigned)ih < (unsigned)g.H) {
+            const float *row = xp + (size_t)ih * g.W;
+            if (VEC) {
+                // pl == 1: columns q0-1 .. q0+KW+1; q0 .. q0+3 are one aligned float4
+                if (iw0 >= 0) v[0] = __ldg(row + iw0);
+                if (q0 + 3 < g.W) {
+                    const float4 m = __ldg(reinterpret_cast<const float4 *>(row + q0));
+                    v[1] = m.x; v[2] = m.y; v[3] = m.z; v[4] = m.w;
+                } else {
+#pragma unroll
+                    for (int k = 1; k < 5; ++k) if (iw0 + k < g.W) v[k] = __ldg(row + iw0 + k);
+                }
+#pragma unroll
+                for (int k = 5; k < WIN; ++k) if (iw0 + k < g.W) v[k] = __ldg(row + iw0 + k);
+            } else {
+#pragma unroll
+                for (int k = 0; k < WIN; ++k) if ((unsigned)(iw0 + k) < (unsigned)g.W) v[k] = __ldg(row + iw0 + k);
+            }
+        }
+        // input row rr is filter row rr of output row p0 and filter row rr-1 of output row p0+1
+#pragma unroll
+        for (int s = 0; s < KW; ++s) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (rr < KH) acc0[j] = fmaf(v[j + s], w[rr * KW + s], acc0[j]);
+                if (rr >= 1) acc1[j] = fmaf(v[j + s], w[(rr - 1) * KW + s], acc1[j]);
+            }
+        }
+    }
+    float *yp = Y + ((size_t)plane * g.P + p0) * g.Q + q0;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        float *a = k ? acc1 : acc0;
+        if (p0 + k >= g.P) break;
+        if (g.relu) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) a[j] = a[j] > 0.f ? a[j] : 0.f;
+        }
+        float *yr = yp + (size_t)k * g.Q;
+        if (VEC && q0 + 3 < g.Q) {
+            *reinterpret_cast<float4 *>(yr) = make_float4(a[0], a[1], a[2], a[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if (q0 + j < g.Q) yr[j] = a[j];
+        }
+    }
+}
+
+template <int KH, int KW>
+int launch_depthwise_unit(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y, cudaStream_t st) {
+    const unsigned Q4 = (unsigned)((g.Q + 3) / 4), P2 = (unsigned)((g.P + 1) / 2);
+    const long long items = (long long)g.N * g.C * P2 * Q4;
+    const unsigned blocks = (unsigned)((items + 255) / 256);
+    // aligned 16-byte accesses: every input and output row starts on a 16-byte boundary
+    const bool vec = g.pl == 1 && g.W % 4 == 0 && g.Q % 4 == 0 &&
+                     (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15) == 0;
+    if (vec)
+        conv2d_depthwise_unit_kernel<KH, KW, true><<<blocks, 256, 0, st>>>(g, X, W, B, Y, (unsigned)items, Q4, P2,
+                                                                            1.0 / (double)Q4, 1.0 / (double)P2);
+    else
+        conv2d_depthwise_unit_kernel<KH, KW, false><<<blocks, 256, 0, st>>>(g, X, W, B, Y, (unsigned)items, Q4, P2,
+                                                                             1.0 / (double)Q4, 1.0 / (double)P2);
+    count_launch();
+    return (int)cudaGetLastError();
+}
+
+bool depthwise_unit_fits(const ConvGeom &g) {
+    if (!(g.Cg == 1 && g.Mg == 1 && g.sh == 1 && g.sw == 1 && g.dh == 1 && g.dw == 1)) return false;
+    if (!((g.kH == 3 && g.kW == 3) || (g.kH == 5 && g.kW == 5))) return false;
+    const long long items = (long long)g.N * g.C * ((g.P + 1) / 2) * ((g.Q + 3) / 4);
+    return items < (1LL << 31) - 256;
+}
+
 void depthwise_window(const ConvGeom &g, int &rows, int &cols, int &pitch) {
     rows = (kDwTP - 1) * g.sh + (g.kH - 1) * g.dh + 1;
     cols = (kDwTQ - 1) * g.sw + (g.kW - 1) * g.dw + 1;
@@ -259,6 +373,10 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
 
 int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
                           void *stream) {
+    if (depthwise_unit_fits(g)) {
+        if (g.kH == 3) return launch_depthwise_unit<3, 3>(g, X, W, B, Y, (cudaStream_t)stream);
+        return launch_depthwise_unit<5, 5>(g, X, W, B, Y, (cudaStream_t)stream);
+    }
     int rows, cols, pitch;
     depthwise_window(g, rows, cols, pitch);
     const int q_tiles = (g.Q + kDwTQ - 1) / kDwTQ, p_tiles = (g.P + kDwTP - 1) / kDwTP;

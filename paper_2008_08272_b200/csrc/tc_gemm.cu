@@ -4,15 +4,17 @@
 // It serves ONNX Gemm (Sec. 3.4.3) and every 1x1, stride-1 convolution (Sec. 4.1),
 // which in NCHW is one GEMM per image: Y[n] (Cout x HW) = W (Cout x C) * X[n] (C x HW).
 //
-// Pipeline (one persistent CTA per SM, 192 threads):
+// Pipeline (one persistent CTA per SM, 320 threads):
 //   warp 0    TMA producer: fp32 operand tiles, 128-byte swizzled, into a ring of
-//             shared-memory stages, completion signalled on mbarriers;
+//             shared-memory stages, completion signalled on mbarriers; the boxes of a
+//             stage are issued by as many lanes at once;
 //   warp 1    one thread issues tcgen05.mma kind::tf32 (128 x BN x 8 per instruction) into
 //             one of two TMEM accumulators and commits stage releases to mbarriers;
-//   warps 2-5 epilogue: tcgen05.ld the finished accumulator (while the MMA warp fills the
+//   warps 2-9 epilogue: tcgen05.ld the finished accumulator (while the MMA warp fills the
 //             other one), apply alpha / beta*C / bias / Relu, stage 32x32 blocks in swizzled
 //             shared memory and write them with TMA stores (plain stores when Y cannot be
-//             described by a tensor map).
+//             described by a tensor map).  Two warps share each TMEM lane quarter and split
+//             its columns, so that a scheduler has a second warp to run while one waits.
 // Either operand may be K-major (reduction index contiguous) or MN-major (row/column
 // index contiguous, e.g. the pixels of an NCHW image); no transposed copy is ever made.
 #include <cuda.h>
@@ -34,10 +36,11 @@ constexpr int kBM = 128;            // UMMA M: rows of D per tile (TMEM lanes)
 constexpr int kBK = 32;             // fp32 elements per stage along K (one 128-byte swizzle row)
 constexpr int kMaxBN = 256;         // UMMA N limit
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
 constexpr int kABytes = kBM * kBK * 4;             // 16 KB
 constexpr int kStoreBufBytes = 32 * 32 * 4;        // one 32x32 fp32 block
-constexpr int kStagingBytes = 4 * 2 * kStoreBufBytes;
+constexpr int kStagingBytes = kEpiWarps * kStoreBufBytes;   // one block per epilogue warp
 constexpr int kBarrierBytes = 256;
 constexpr int kSmemLimit = 232448;                 // 227 KB opt-in maximum per CTA
 
@@ -95,7 +98,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full[a], 1);
-            mbar_init(&tmem_empty[a], 4);
+            mbar_init(&tmem_empty[a], kEpiWarps);
         }
         mbar_fence_init();
         prefetch_tmap(&tmA);
@@ -115,31 +118,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (elect_one()) {
+        // The whole warp runs the loop: a stage's copies (one box for a K-major operand, one per 32
+        // rows/columns for an MN-major one, up to 12 in all) are issued by as many lanes at once.  A
+        // single thread pays its full instruction latency for every box and cannot keep the ring full.
+        {
             int stage = 0;
             uint32_t phase = 0;
+            const int na = p.a_mn ? kBM / 32 : 1, nb = p.b_mn ? p.BN / 32 : 1;
+            // this lane's box: lanes [0, na) load A pieces, lanes [na, na + nb) load B pieces
+            const bool is_a = lane < na, is_b = !is_a && lane < na + nb;
+            const int j = is_a ? lane : lane - na;
+            const uint32_t dst_off = is_a ? (uint32_t)j * 4096u : (uint32_t)kABytes + (uint32_t)j * 4096u;
             for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
                 const int tm = t % p.tiles_m;
                 const int tn = (t / p.tiles_m) % p.tiles_n;
                 const int b = t / (p.tiles_m * p.tiles_n);
                 const int ab = p.a_batched ? b : 0, bb = p.b_batched ? b : 0;
+                // coordinates of this lane's box at k-block 0 (c0 = contiguous axis) and their step per k-block
+                int c0, c1, d0, d1;
+                if (is_a) {
+                    if (!p.a_mn) { c0 = 0; c1 = tm * kBM; d0 = kBK; d1 = 0; }
+                    else { c0 = tm * kBM + j * 32; c1 = 0; d0 = 0; d1 = kBK; }
+                } else {
+                    if (!p.b_mn) { c0 = 0; c1 = tn * p.BN; d0 = kBK; d1 = 0; }
+                    else { c0 = tn * p.BN + j * 32; c1 = 0; d0 = 0; d1 = kBK; }
+                }
+                const int c2 = is_a ? ab : bb;
+                const CUtensorMap *tmap = is_a ? &tmA : &tmB;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
-                    mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
-                    uint8_t *sA = stages + (size_t)stage * p.stage_bytes;
-                    uint8_t *sB = sA + kABytes;
-                    if (!p.a_mn) {
-                        tma_load_3d(sA, &tmA, &full[stage], kb * kBK, tm * kBM, ab);
-                    } else {
-                        for (int j = 0; j < kBM / 32; ++j)
-                            tma_load_3d(sA + j * 4096, &tmA, &full[stage], tm * kBM + j * 32, kb * kBK, ab);
-                    }
-                    if (!p.b_mn) {
-                        tma_load_3d(sB, &tmB, &full[stage], kb * kBK, tn * p.BN, bb);
-                    } else {
-                        for (int j = 0; j < p.BN / 32; ++j)
-                            tma_load_3d(sB + j * 4096, &tmB, &full[stage], tn * p.BN + j * 32, kb * kBK, bb);
-                    }
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
+                    __syncwarp();
+                    if (is_a || is_b)
+                        tma_load_3d(stages + (size_t)stage * p.stage_bytes + dst_off, tmap, &full[stage], c0, c1, c2);
+                    c0 += d0;
+                    c1 += d1;
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -149,6 +162,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (elect_one()) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
+            // Descriptor words that do not change: everything but the 14-bit start address.
+            // K-major: 32 bytes further along the swizzled 128-byte rows per instruction (8-row groups
+            // 1024 bytes apart).  MN-major 32-bit operands use the 128-byte swizzle with 32-byte atoms:
+            // atoms of four 128-byte K rows (512 bytes apart along K), blocks of 32 rows/columns 4096
+            // bytes apart; one instruction consumes eight K rows (1024 bytes).
+            const uint64_t a_tmpl = p.a_mn ? make_smem_desc(0, 4096, 512, kSwizzle128B32) : make_smem_desc(0, 16, 1024, kSwizzle128B);
+            const uint64_t b_tmpl = p.b_mn ? make_smem_desc(0, 4096, 512, kSwizzle128B32) : make_smem_desc(0, 16, 1024, kSwizzle128B);
+            const uint32_t a_hi = (uint32_t)(a_tmpl >> 32), b_hi = (uint32_t)(b_tmpl >> 32);
+            const uint32_t a_lo_c = (uint32_t)a_tmpl, b_lo_c = (uint32_t)b_tmpl;
+            const uint32_t a_k16 = (p.a_mn ? 1024u : 32u) >> 4, b_k16 = (p.b_mn ? 1024u : 32u) >> 4;
+            const uint32_t idesc = p.idesc;
             GP_DECL;
             for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
                 mbar_wait(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
@@ -160,19 +184,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tc_fence_after_sync();
                     GP_MARK(1);
                     const uint32_t sA = smem_u32(stages + (size_t)stage * p.stage_bytes);
-                    const uint32_t sB = sA + kABytes;
+                    const uint32_t a16 = sA >> 4, b16 = (sA + kABytes) >> 4;
                     const int k_left = p.K - kb * kBK;
                     const int k8 = k_left >= kBK ? kBK / 8 : (k_left + 7) / 8;
-                    for (int k = 0; k < k8; ++k) {
-                        // K-major: 32 bytes further along the swizzled 128-byte rows (8-row groups
-                        // 1024 bytes apart).  MN-major 32-bit operands use the 128-byte swizzle with
-                        // 32-byte atoms: atoms of four 128-byte K rows (512 bytes apart along K), blocks
-                        // of 32 rows/columns 4096 bytes apart; one instruction consumes eight K rows.
-                        const uint64_t ad = p.a_mn ? make_smem_desc(sA + k * 1024, 4096, 512, kSwizzle128B32)
-                                                   : make_smem_desc(sA + k * 32, 16, 1024, kSwizzle128B);
-                        const uint64_t bd = p.b_mn ? make_smem_desc(sB + k * 1024, 4096, 512, kSwizzle128B32)
-                                                   : make_smem_desc(sB + k * 32, 16, 1024, kSwizzle128B);
-                        mma_tf32(d_tmem, ad, bd, p.idesc, (kb | k) != 0);
+                    // one thread issues everything: keep the per-instruction work to two adds
+#pragma unroll
+                    for (int k = 0; k < kBK / 8; ++k) {
+                        if (k < k8)
+                            mma_tf32_lohi(d_tmem, a_lo_c | ((a16 + (uint32_t)k * a_k16) & 0x3FFFu), a_hi,
+                                          b_lo_c | ((b16 + (uint32_t)k * b_k16) & 0x3FFFu), b_hi, idesc, (kb | k) != 0);
                     }
                     mma_commit(&empty[stage]);
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
@@ -187,9 +207,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;                    // TMEM lane quarter this warp may read
-        uint8_t *my_staging = staging + q * 2 * kStoreBufBytes;
+        const int half = (warp - 2) >> 2;          // which half of the tile's 32-column blocks
+        uint8_t *buf = staging + (warp - 2) * kStoreBufBytes;
         int acc = 0;
-        uint32_t acc_phase = 0, store_idx = 0;
+        uint32_t acc_phase = 0;
         GP_DECL;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const int tm = t % p.tiles_m;
@@ -202,7 +223,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int row = row0 + lane;
             if (row0 < p.M) {
                 const float rb = (p.row_bias && row < p.M) ? __ldg(p.row_bias + row) : 0.f;
-                const int nchunk = min(p.BN / 32, (p.N - tn * p.BN + 31) / 32);
+                const int nchunk_all = min(p.BN / 32, (p.N - tn * p.BN + 31) / 32);
+                const int c_lo = half ? (nchunk_all + 1) / 2 : 0, c_hi = half ? nchunk_all : (nchunk_all + 1) / 2;
                 const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBN);
                 // one 32x32 block: scale, add, activate, hand to the store path
                 auto finish = [&](const uint32_t (&v)[32], int chunk) {
@@ -230,10 +252,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     GP_MARK(2);
                     // Stage the 32x32 block in shared memory, row `lane`, 16-byte chunk c at position
                     // c ^ (lane % 8) (the 128-byte swizzle, conflict-free for these 16-byte stores).
-                    uint8_t *buf = my_staging + (store_idx & 1) * kStoreBufBytes;
-                    ++store_idx;
                     if (p.y_tma) {
-                        if (lane == 0) tma_store_wait_read<1>();   // the store that last read this buffer is done
+                        if (lane == 0) tma_store_wait_read<0>();   // the store that last read this buffer is done
                     }
                     __syncwarp();
                     GP_MARK(3);
@@ -275,15 +295,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // TMEM reads are software-pipelined: the next block's load is in flight while
                 // the current one is finished and stored
                 uint32_t va[32], vb[32];
-                tmem_ld_32x32(tbase, va);
-                for (int chunk = 0; chunk < nchunk; chunk += 2) {
+                if (c_lo < c_hi) tmem_ld_32x32(tbase + (uint32_t)(c_lo * 32), va);
+                for (int chunk = c_lo; chunk < c_hi; chunk += 2) {
                     tmem_ld_wait();
-                    if (chunk + 1 < nchunk) tmem_ld_32x32(tbase + (uint32_t)((chunk + 1) * 32), vb);
+                    if (chunk + 1 < c_hi) tmem_ld_32x32(tbase + (uint32_t)((chunk + 1) * 32), vb);
                     GP_MARK(1);
                     finish(va, chunk);
-                    if (chunk + 1 < nchunk) {
+                    if (chunk + 1 < c_hi) {
                         tmem_ld_wait();
-                        if (chunk + 2 < nchunk) tmem_ld_32x32(tbase + (uint32_t)((chunk + 2) * 32), va);
+                        if (chunk + 2 < c_hi) tmem_ld_32x32(tbase + (uint32_t)((chunk + 2) * 32), va);
                         GP_MARK(1);
                         finish(vb, chunk + 1);
                     }
