@@ -120,9 +120,14 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
-// arrive on an mbarrier of another CTA of the cluster (address from map_to_cta)
+// Arrive on an mbarrier of another CTA of the cluster (address from map_to_cta).  Relaxed: a release
+// at cluster scope stalls the thread for about a thousand cycles, and nothing here needs it.  What
+// the arrival announces sits in shared memory and has already been ordered for its consumer: either
+// an asynchronous copy whose completion the announcing thread has observed on its own barrier, or
+// writes followed by a proxy fence, or TMEM reads closed by tcgen05.fence::before_thread_sync.  The
+// consumer acquires at cluster scope.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // every thread of every CTA of the cluster
 __device__ __forceinline__ void cluster_sync_all() {

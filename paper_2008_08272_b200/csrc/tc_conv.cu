@@ -408,7 +408,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                     if (i < nu) {
                         const int u = xt + i * kXformThreads;
                         const int ch = conv_fdiv(u, per_stage_slots, g.inv_pss), idx = u - ch * per_stage_slots;
-                        udst[i] = (uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u;
+                        // operand rows are 16 bytes apart: the low four bits carry the unit's chunk index
+                        udst[i] = ((uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u) | (uint32_t)ch;
                         const int pl = conv_fdiv(idx, g.SLOTS, g.inv_SLOTS), j = idx - pl * g.SLOTS;
                         const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
                         if (Gs < (uint32_t)g.total_slots) {
@@ -446,43 +447,28 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 uint8_t *adst = a_st + (size_t)as * g.a_stage_bytes;
                 const int cbx = cb + rot < ncb ? cb + rot : cb + rot - ncb;
                 const int c_left = g.Cg - cbx * KB;    // channels of this block that exist
-                if (c_left >= KB) {
-                    // every channel of the block exists: all reads first, then round and store
+                {
+                    // all reads first (independent, so their latencies overlap), then round and store;
+                    // channels past the end of the group (last block only) read as zero
                     float v[kOwned][4];
 #pragma unroll
                     for (int i = 0; i < kOwned; ++i) {
                         v[i][0] = v[i][1] = v[i][2] = v[i][3] = 0.f;
                         if (i < nu && uoff[i] >= 0) {
                             const float *r = raw + uoff[i];
-                            v[i][0] = r[0];
-                            v[i][1] = r[cp];
-                            v[i][2] = r[2 * cp];
-                            v[i][3] = r[3 * cp];
+                            const int left = c_left - (int)(udst[i] & 15u) * 4;
+                            if (left > 0) v[i][0] = r[0];
+                            if (left > 1) v[i][1] = r[cp];
+                            if (left > 2) v[i][2] = r[2 * cp];
+                            if (left > 3) v[i][3] = r[3 * cp];
                         }
                     }
 #pragma unroll
                     for (int i = 0; i < kOwned; ++i)
                         if (i < nu)
-                            *reinterpret_cast<float4 *>(adst + udst[i]) =
+                            *reinterpret_cast<float4 *>(adst + (udst[i] & ~15u)) =
                                 make_float4(round_tf32(v[i][0]), round_tf32(v[i][1]), round_tf32(v[i][2]),
                                             round_tf32(v[i][3]));
-                } else {
-#pragma unroll
-                    for (int i = 0; i < kOwned; ++i) {
-                        if (i < nu) {
-                            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (uoff[i] >= 0) {
-                                const float *r = raw + uoff[i];
-                                const int ch = (xt + i * kXformThreads) / per_stage_slots;
-                                const int left = c_left - ch * 4;
-                                if (left > 0) v.x = round_tf32(r[0]);
-                                if (left > 1) v.y = round_tf32(r[cp]);
-                                if (left > 2) v.z = round_tf32(r[2 * cp]);
-                                if (left > 3) v.w = round_tf32(r[3 * cp]);
-                            }
-                            *reinterpret_cast<float4 *>(adst + udst[i]) = v;
-                        }
-                    }
                 }
                 PROF_MARK(2);
                 fence_proxy_async_smem();
@@ -613,7 +599,7 @@ int pick_conv_bn(int Mg) {
     return best;
 }
 
-bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, TcConvPlan &g) {
+bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &g) {
     if (ctas == 2 && BN % 16) return false;      // M = 256 instructions take N in multiples of 16
     g.ctas = ctas;
     g.BNH = BN / ctas;
@@ -640,7 +626,8 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, TcConvPlan &g) {
     g.MT = MT; g.BN = BN;
     g.ctiles = (c.Mg + BN - 1) / BN;
     const long long slots = (long long)MT * 128 + maxshift;
-    if (slots * g.planes * (c.Cg >= 16 ? 4 : 1) > kOwned * kXformThreads) return false;
+    if (c.Cg < 16) KB = 4;
+    if (slots * g.planes * (KB / 4) > kOwned * kXformThreads) return false;
     g.SLOTS = (int)slots;
     if ((g.SLOTS + L - 2) / L + 1 > kConvMaxSeg) return false;
     g.plane_pitch = g.SLOTS * 16;
@@ -661,13 +648,16 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, TcConvPlan &g) {
 
     // K-steps of one channel block
     if (c.Cg >= 16) {
-        g.KB = 16;
-        g.n_steps = 2 * g.taps;
+        // blocks of KB = 16, 32 or 64 channels: KB/8 steps per tap, step j reading chunks 2j and 2j+1
+        const int spt = KB / 8;
+        g.KB = KB;
+        g.n_steps = spt * g.taps;
+        if (g.n_steps > kConvMaxSteps) return false;
         const uint32_t lbo16 = (uint32_t)g.chunk_pitch >> 4;
-        if (lbo16 >= (1u << 14)) return false;
+        if ((uint32_t)(KB / 4) * lbo16 >= (1u << 14)) return false;     // every chunk start must fit the address field
         for (int tp = 0; tp < g.taps; ++tp)
-            for (int j = 0; j < 2; ++j) {
-                const int s = 2 * tp + j;
+            for (int j = 0; j < spt; ++j) {
+                const int s = spt * tp + j;
                 g.step_a[s] = ((uint32_t)tap_off16[tp] + (uint32_t)j * 2u * lbo16) | (lbo16 << 16);
                 g.src_tap[s][0] = g.src_tap[s][1] = (short)tp;
                 g.src_c0[s][0] = (short)(j * 8);
@@ -792,32 +782,33 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
     const int sms = 148;
     const int bn0 = pick_conv_bn(c.Mg);
     // candidate tiles (CTAs per tile, accumulators per CTA, channels per tile)
-    int cand[16][3];
+    int cand[48][4];
     int ncand = 0;
-    auto add = [&](int ctas, int mt, int bn) {
+    auto add = [&](int ctas, int mt, int bn, int kb) {
         for (int i = 0; i < ncand; ++i)
-            if (cand[i][0] == ctas && cand[i][1] == mt && cand[i][2] == bn) return;
-        cand[ncand][0] = ctas; cand[ncand][1] = mt; cand[ncand][2] = bn; ++ncand;
+            if (cand[i][0] == ctas && cand[i][1] == mt && cand[i][2] == bn && cand[i][3] == kb) return;
+        cand[ncand][0] = ctas; cand[ncand][1] = mt; cand[ncand][2] = bn; cand[ncand][3] = kb; ++ncand;
     };
-    int fc = 0, fm = 0, fb = 0;
-    if (const char *e = getenv("ONNXB_CONV_TILE")) {      // "ctas,MT,BN": pin the tile for A/B measurements
-        if (sscanf(e, "%d,%d,%d", &fc, &fm, &fb) == 3 && (fc == 1 || fc == 2) && (fm == 1 || fm == 2) && fb >= 16 &&
-            fb <= 256 && fb % 16 == 0)
-            add(fc, fm, fb);
+    int fc = 0, fm = 0, fb = 0, fk = 16;
+    if (const char *e = getenv("ONNXB_CONV_TILE")) {      // "ctas,MT,BN[,KB]": pin the tile for A/B measurements
+        if (sscanf(e, "%d,%d,%d,%d", &fc, &fm, &fb, &fk) >= 3 && (fc == 1 || fc == 2) && (fm == 1 || fm == 2) &&
+            fb >= 16 && fb <= 256 && fb % 16 == 0 && (fk == 16 || fk == 32 || fk == 64))
+            add(fc, fm, fb, fk);
     }
     if (ncand == 0) {
-        for (int ctas = 2; ctas >= 1; --ctas) {
-            add(ctas, 2, bn0);
-            add(ctas, 1, bn0);
-            if (bn0 > 128) { add(ctas, 2, 128); add(ctas, 1, 128); }
-            if (bn0 > 64) add(ctas, 1, 64);
-        }
+        for (int kb = 16; kb <= 64 && (kb == 16 || kb <= c.Cg); kb *= 2)
+            for (int ctas = 2; ctas >= 1; --ctas) {
+                add(ctas, 2, bn0, kb);
+                add(ctas, 1, bn0, kb);
+                if (bn0 > 128) { add(ctas, 2, 128, kb); add(ctas, 1, 128, kb); }
+                if (bn0 > 64) add(ctas, 1, 64, kb);
+            }
     }
     bool have = false;
     double best_cost = 0;
     for (int i = 0; i < ncand; ++i) {
         TcConvPlan p;
-        if (!fill_plan(c, cand[i][0], cand[i][1], cand[i][2], p)) continue;
+        if (!fill_plan(c, cand[i][0], cand[i][1], cand[i][2], cand[i][3], p)) continue;
         // Cost in SM cycles per CTA, fitted to measured tile sweeps of the ResNet-50 3x3 layers.  Per
         // channel block the slowest of: the tensor pipe (BN/2 cycles per 128 x BN x 8 share of an
         // instruction, or the 128 bytes/cycle of shared memory its operands need, whichever is longer),
@@ -834,7 +825,10 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
         const double w_bytes = (double)p.n_steps * p.b_step_bytes;
         const double slots16 = (double)p.planes * p.SLOTS * 16.0 * p.nchunks;
         const double t_smem = (n_inst * op_bytes + w_bytes + 3.0 * slots16) / 90.0;
-        const double t_w = w_bytes / std::min(48.0, 3600.0 / active);
+        // the weight ring must also cover the latency of its copies (about 2500 cycles from issue to
+        // landing under load): a ring holding less than that much of the stream paces the block
+        const double ring = (double)p.nb_stages * p.b_stage_bytes;
+        const double t_w = std::max(w_bytes / std::min(48.0, 3600.0 / active), w_bytes * 2500.0 / ring);
         const double t_x = 300.0 + 100.0 * ((p.planes * p.SLOTS * p.nchunks + 255) / 256);
         const double per_cb = std::max(std::max(t_mma, t_smem), std::max(t_w, t_x)) + 400.0 + (p.ctas == 2 ? 700.0 : 0.0);
         const bool dbl = p.MT == 1 || p.BN <= 128;
