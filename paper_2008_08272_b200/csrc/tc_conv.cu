@@ -64,10 +64,10 @@ static_assert(sizeof(Bars) <= kBarBytes, "barrier block too large");
 
 #ifdef ONNXB_PROFILE
 __device__ long long g_prof[148 * 16];
-#define PROF_DECL long long pt_ = clock64(), pacc_[5] = {0, 0, 0, 0, 0}
+#define PROF_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
 #define PROF_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
 #define PROF_RESET() do { pt_ = clock64(); } while (0)
-#define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 5; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
+#define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 6; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
 // event log of CTA 0: kind k (0..7), sequence number i (0..63) -> clock
 __device__ long long g_log[8 * 64];
 #define LOG(k, i) do { if (blockIdx.x == 0 && (i) < 64) g_log[(k) * 64 + (i)] = clock64(); } while (0)
@@ -98,17 +98,20 @@ __device__ long long g_chk[8];
 // i.e. for each K-step the exact shared-memory image of one CTA's part of the K-major B operand: two
 // 16-byte chunks (4 reduction terms each) per output channel, rows 16 bytes apart.  Values are rounded to TF32 (nearest);
 // rows past the group's channels, channels past Cg and unpaired taps are zero.
+// Launched with programmatic stream serialization: it may become resident while the previous kernel
+// of the stream drains, and waits (pdl_wait) before it touches W or the workspace.
 __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict__ W, float4 *__restrict__ out) {
     pdl_launch_dependents();
-    const long long total = g.packed_floats / 4;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        long long t = i;
-        const int row = (int)(t % g.BNH); t /= g.BNH;
-        const int k = (int)(t % 2); t /= 2;
-        const int step = (int)(t % g.n_steps); t /= g.n_steps;
-        const int cb = (int)(t % g.ncb); t /= g.ncb;
-        const int ct = (int)(t % (g.ctiles * g.ctas)); t /= g.ctiles * g.ctas;   // BNH-wide tile: (tile, CTA of the pair)
+    const unsigned total = (unsigned)(g.packed_floats / 4);          // the planner keeps this below 2^31
+    pdl_wait();
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        unsigned t = i;
+        const int row = (int)(t % (unsigned)g.BNH); t /= (unsigned)g.BNH;
+        const int k = (int)(t & 1u); t >>= 1;
+        const int step = (int)(t % (unsigned)g.n_steps); t /= (unsigned)g.n_steps;
+        const int cb = (int)(t % (unsigned)g.ncb); t /= (unsigned)g.ncb;
+        const unsigned cts = (unsigned)(g.ctiles * g.ctas);
+        const int ct = (int)(t % cts); t /= cts;                     // BNH-wide tile: (tile, CTA of the pair)
         const int grp = (int)t;
         const int mg = ct * g.BNH + row;
         const int tap = g.src_tap[step][k];
@@ -399,6 +402,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 // per-thread offsets of the tile, from its segment table (ready before the data)
                 const uint32_t sp = tile_it & 1u;
                 mbar_wait(&bars->seg_full[sp], (tile_it >> 1) & 1u, err, 21);
+                PROF_MARK(4);
                 ++tile_it;
                 const TcConvSegs *segs = reinterpret_cast<const TcConvSegs *>(seg_st + sp * kSegBytes);
 #pragma unroll
@@ -407,24 +411,28 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                     udst[i] = 0;
                     if (i < nu) {
                         const int u = xt + i * kXformThreads;
-                        const int ch = conv_fdiv(u, per_stage_slots, g.inv_pss), idx = u - ch * per_stage_slots;
+                        const int ch = conv_fdiv(u, g.planes * g.SLOTS, g.dv_pss), idx = u - ch * per_stage_slots;
                         // operand rows are 16 bytes apart: the low four bits carry the unit's chunk index
                         udst[i] = ((uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u) | (uint32_t)ch;
-                        const int pl = conv_fdiv(idx, g.SLOTS, g.inv_SLOTS), j = idx - pl * g.SLOTS;
+                        const int pl = conv_fdiv(idx, g.SLOTS, g.dv_SLOTS), j = idx - pl * g.SLOTS;
                         const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
                         if (Gs < (uint32_t)g.total_slots) {
-                            const int n = conv_fdiv((int)Gs, g.L, g.inv_L);
+                            const int n = conv_fdiv((int)Gs, g.L, g.dv_L);
                             const int uu = (int)Gs - n * g.L;
-                            const int hq = conv_fdiv(uu, g.Ws, g.inv_Ws), wq = uu - hq * g.Ws;
-                            const int h = hq * g.sh + g.pa[pl] - g.pt;
-                            const int w = wq * g.sw + g.pb[pl] - g.pl;
+                            const int hq = conv_fdiv(uu, g.Ws, g.dv_Ws), wq = uu - hq * g.Ws;
+                            // fixed-index reads of the parity tables (a dynamic index into kernel
+                            // parameters costs an indexed constant load per use)
+                            const int pa = pl == 0 ? g.pa[0] : pl == 1 ? g.pa[1] : pl == 2 ? g.pa[2] : g.pa[3];
+                            const int pb = pl == 0 ? g.pb[0] : pl == 1 ? g.pb[1] : pl == 2 ? g.pb[2] : g.pb[3];
+                            const int h = hq * g.sh + pa - g.pt;
+                            const int w = wq * g.sw + pb - g.pl;
                             const int sg = n - segs->n_first;
                             if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
                                 const int f = h * g.W + w - segs->f0[sg];
                                 int o;
                                 if (g.raw_mode == 1) o = segs->base[sg] + f;
                                 else {
-                                    const int bx = conv_fdiv(f, g.BOXP, g.inv_BOXP);
+                                    const int bx = conv_fdiv(f, g.BOXP, g.dv_BOXP);
                                     o = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
                                 }
                                 uoff[i] = o + ch * 4 * cp;
@@ -434,7 +442,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars->seg_empty[sp]);
-                PROF_MARK(2);
+                PROF_MARK(5);
             }
             for (int cb = 0; cb < ncb; ++cb) {
                 mbar_wait(&bars->raw_full[rs], rphase, err, 16);
@@ -710,6 +718,7 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
     g.spb = std::max(1, std::min(std::min(g.n_steps, kMaxSpb), 32768 / g.b_step_bytes));   // several K-steps per weight stage
     g.idesc = tc::make_idesc_tf32(128 * ctas, BN, 0, 0);
     g.packed_floats = (long long)c.group * g.ctiles * g.ncb * g.n_steps * BN * 8;     // both CTAs' parts
+    if (g.packed_floats >= (1LL << 32)) return false;                                  // 32-bit indexing in the packing kernel
     // raw stage size: widest flat pixel range any tile needs, found by walking the tiles
     g.BOXP = 256;
     const long long walk = std::min<long long>(ptiles, L + 2);
@@ -761,11 +770,11 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
     g.b_stage_bytes = g.spb * g.b_step_bytes;
     if (room < 2LL * g.b_stage_bytes) return false;
     g.nb_stages = (int)std::min<long long>(kMaxBStages, room / g.b_stage_bytes);
-    g.inv_L = conv_recip(g.L);
-    g.inv_Ws = conv_recip(g.Ws);
-    g.inv_BOXP = conv_recip(g.BOXP);
-    g.inv_SLOTS = conv_recip(g.SLOTS);
-    g.inv_pss = conv_recip(g.planes * g.SLOTS);
+    g.dv_L = conv_divisor(g.L);
+    g.dv_Ws = conv_divisor(g.Ws);
+    g.dv_BOXP = conv_divisor(g.BOXP);
+    g.dv_SLOTS = conv_divisor(g.SLOTS);
+    g.dv_pss = conv_divisor(g.planes * g.SLOTS);
     return true;
 }
 
@@ -904,9 +913,9 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     {
         const long long vec = plan.packed_floats / 4;
         const int blocks = (int)std::min<long long>((vec + 255) / 256, 148 * 16);
-        pack_weights_kernel<<<blocks, 256, 0, st>>>(plan, W, reinterpret_cast<float4 *>(workspace));
+        const cudaError_t e = launch_pdl(pack_weights_kernel, dim3(blocks), dim3(256), 0, st, plan, W,
+                                         reinterpret_cast<float4 *>(workspace));
         count_launch();
-        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return (int)e;
     }
     // 2. the convolution

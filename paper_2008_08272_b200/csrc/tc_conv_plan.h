@@ -26,6 +26,10 @@ constexpr int kConvMaxTaps = 64;
 constexpr int kConvMaxSteps = 128;     // MMA K-steps (8 reduction terms each) per channel block
 constexpr int kConvMaxSeg = 8;
 
+struct ConvDivisor {
+    uint32_t d, m, s1, s2;
+};
+
 struct TcConvPlan {
     // problem
     int N, C, H, W, M, Cg, Mg, kH, kW, P, Q, pt, pl, sh, sw, dh, dw, group, relu;
@@ -61,23 +65,35 @@ struct TcConvPlan {
     int chunk_pitch, plane_pitch;    // bytes between 4-channel chunks / parity planes inside an A stage
     uint32_t idesc;
     long long packed_floats;         // size of the packed weight buffer
-    // reciprocals (nudged up by 2^-40) of the divisors device code needs per slot: see conv_fdiv
-    double inv_L, inv_Ws, inv_BOXP, inv_SLOTS, inv_pss;
+    // divisors device code needs per slot, as multiply-and-shift constants (see conv_fdiv)
+    ConvDivisor dv_L, dv_Ws, dv_BOXP, dv_SLOTS, dv_pss;
 };
 
-// floor(n / d) for 0 <= n < 2^31.  On the device: one double multiply by the stored reciprocal
-// (exact: the nudge keeps the product at or above the true quotient and the overshoot stays below
-// 1/d); on the host: plain integer division.
-ONNXB_HD inline int conv_fdiv(int n, int d, double inv) {
+// floor(n / d) for any 32-bit unsigned n.  On the device: the round-up multiply-and-shift method
+// (Granlund and Montgomery, "Division by invariant integers using multiplication"): with
+// l = ceil(log2 d) and m = floor(2^32 (2^l - d) / d) + 1, t = high32(m * n) and
+// q = (t + ((n - t) >> min(l, 1))) >> max(l - 1, 0).  On the host: plain division.
+// (The host passes the divisor itself: while a plan is being filled its constants are not yet set.)
+ONNXB_HD inline int conv_fdiv(int n, int d, const ConvDivisor &dv) {
 #if defined(__CUDA_ARCH__)
     (void)d;
-    return __double2int_rd((double)n * inv);
+    const uint32_t un = (uint32_t)n, t = __umulhi(dv.m, un);
+    return (int)((t + ((un - t) >> dv.s1)) >> dv.s2);
 #else
-    (void)inv;
-    return n / d;
+    (void)dv;
+    return (int)((uint32_t)n / (uint32_t)d);
 #endif
 }
-inline double conv_recip(int d) { return (1.0 / (double)d) * (1.0 + 1.0 / 1099511627776.0); }
+inline ConvDivisor conv_divisor(int d) {
+    ConvDivisor dv;
+    dv.d = (uint32_t)d;
+    int l = 0;
+    while ((1ull << l) < (unsigned long long)d) ++l;
+    dv.m = (uint32_t)(((1ull << 32) * ((1ull << l) - (unsigned long long)d)) / (unsigned long long)d + 1);
+    dv.s1 = l < 1 ? (uint32_t)l : 1u;
+    dv.s2 = l > 1 ? (uint32_t)(l - 1) : 0u;
+    return dv;
+}
 
 struct TcConvSegs {
     int n_first, nseg;
@@ -97,8 +113,8 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
         t.total_floats = 0;
         return;
     }
-    t.n_first = conv_fdiv((int)G0, g.L, g.inv_L);
-    const int n_last = conv_fdiv((int)(Gend - 1), g.L, g.inv_L);
+    t.n_first = conv_fdiv((int)G0, g.L, g.dv_L);
+    const int n_last = conv_fdiv((int)(Gend - 1), g.L, g.dv_L);
     t.nseg = n_last - t.n_first + 1;
     if (t.nseg > kConvMaxSeg) t.nseg = kConvMaxSeg;   // excluded by the planner
     int base = 0;
@@ -107,7 +123,7 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
         const long long lo = G0 > n * g.L ? G0 : n * g.L;
         const long long hi = Gend < (n + 1) * g.L ? Gend : (n + 1) * g.L;
         const int u_lo = (int)(lo - n * g.L), u_hi = (int)(hi - n * g.L);   // [u_lo, u_hi)
-        const int hq_lo = conv_fdiv(u_lo, g.Ws, g.inv_Ws), hq_hi = conv_fdiv(u_hi - 1, g.Ws, g.inv_Ws);
+        const int hq_lo = conv_fdiv(u_lo, g.Ws, g.dv_Ws), hq_hi = conv_fdiv(u_hi - 1, g.Ws, g.dv_Ws);
         int h_min = hq_lo * g.sh + g.a_min - g.pt;
         int h_max = hq_hi * g.sh + g.a_max - g.pt;
         if (h_min < 0) h_min = 0;
@@ -124,7 +140,7 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
             const int f0 = (h_min * g.W) & ~3;
             const int len = (h_max + 1) * g.W - f0;
             t.f0[i] = f0;
-            t.nbox[i] = conv_fdiv(len + g.BOXP - 1, g.BOXP, g.inv_BOXP);
+            t.nbox[i] = conv_fdiv(len + g.BOXP - 1, g.BOXP, g.dv_BOXP);
             base += t.nbox[i] * g.BOXP * g.KB;
         }
     }
