@@ -66,6 +66,11 @@ struct Params {
     long long c_si, c_sj, c_sb;
     const float *row_bias;     // optional per-row addend (convolution bias)
     int relu;
+    // MN-major B in one copy per stage: a 4-D view (32 columns of a block, K row, block of 32 columns,
+    // batch) lets a single box carry all of a tile's 32-column blocks in the order the MMA wants them.
+    int b_big;                 // that view is in use
+    int b_nb_last;             // full blocks in the last column tile (0: none), loaded through tmBt
+    int b_ragged;              // the last column tile ends in a partial block, loaded through tmB
     float *Y;                  // used by the plain-store epilogue
     long long y_ld, y_sb;
     int y_split;               // > 0: columns are groups of y_split, y_group elements apart (plain stores only)
@@ -76,6 +81,7 @@ struct Params {
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmBb, const __grid_constant__ CUtensorMap tmBt,
                const __grid_constant__ CUtensorMap tmY, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler
@@ -103,6 +109,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         mbar_fence_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        if (p.b_big) { prefetch_tmap(&tmBb); prefetch_tmap(&tmBt); }
         if (p.y_tma) prefetch_tmap(&tmY);
     }
     if (warp == 1) {
@@ -118,39 +125,65 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        // The whole warp runs the loop: a stage's copies (one box for a K-major operand, one per 32
-        // rows/columns for an MN-major one, up to 12 in all) are issued by as many lanes at once.  A
-        // single thread pays its full instruction latency for every box and cannot keep the ring full.
+        // The TMA unit spends 70-90 cycles on every copy instruction however small it is, so a stage is
+        // fetched with as few instructions as possible (an MN-major B of up to eight 4 KB blocks through
+        // one 4-D box where the problem allows), and the whole warp runs the loop so that the copies of
+        // a stage are issued by as many lanes at once instead of one thread paying its instruction
+        // latency for each.
         {
             int stage = 0;
             uint32_t phase = 0;
-            const int na = p.a_mn ? kBM / 32 : 1, nb = p.b_mn ? p.BN / 32 : 1;
-            // this lane's box: lanes [0, na) load A pieces, lanes [na, na + nb) load B pieces
+            const int na = p.a_mn ? kBM / 32 : 1;
+            const int nb = !p.b_mn ? 1 : (p.b_big ? 2 : p.BN / 32);
+            // this lane's copy: lanes [0, na) load A pieces, lanes [na, na + nb) load B pieces
             const bool is_a = lane < na, is_b = !is_a && lane < na + nb;
             const int j = is_a ? lane : lane - na;
-            const uint32_t dst_off = is_a ? (uint32_t)j * 4096u : (uint32_t)kABytes + (uint32_t)j * 4096u;
             for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
                 const int tm = t % p.tiles_m;
                 const int tn = (t / p.tiles_m) % p.tiles_n;
                 const int b = t / (p.tiles_m * p.tiles_n);
                 const int ab = p.a_batched ? b : 0, bb = p.b_batched ? b : 0;
                 // coordinates of this lane's box at k-block 0 (c0 = contiguous axis) and their step per k-block
-                int c0, c1, d0, d1;
+                int c0 = 0, c1 = 0, d0 = 0, d1 = 0, kind = 0;      // kind: 0 none, 1 3-D map, 2 big B box, 3 tail B box
+                uint32_t dst_off = 0, tx = 0;
+                const CUtensorMap *tmap = &tmA;
                 if (is_a) {
-                    if (!p.a_mn) { c0 = 0; c1 = tm * kBM; d0 = kBK; d1 = 0; }
-                    else { c0 = tm * kBM + j * 32; c1 = 0; d0 = 0; d1 = kBK; }
-                } else {
-                    if (!p.b_mn) { c0 = 0; c1 = tn * p.BN; d0 = kBK; d1 = 0; }
-                    else { c0 = tn * p.BN + j * 32; c1 = 0; d0 = 0; d1 = kBK; }
+                    kind = 1;
+                    dst_off = (uint32_t)j * 4096u;
+                    if (!p.a_mn) { c1 = tm * kBM; d0 = kBK; }
+                    else { c0 = tm * kBM + j * 32; d1 = kBK; }
+                } else if (is_b) {
+                    tmap = &tmB;
+                    if (!p.b_mn) { kind = 1; dst_off = kABytes; c1 = tn * p.BN; d0 = kBK; }
+                    else if (!p.b_big) { kind = 1; dst_off = (uint32_t)kABytes + (uint32_t)j * 4096u; c0 = tn * p.BN + j * 32; d1 = kBK; }
+                    else {
+                        const bool last = tn == p.tiles_n - 1 && (p.b_nb_last != p.BN / 32 || p.b_ragged);
+                        if (j == 0) {
+                            // all of the tile's full blocks: c0 = first block
+                            if (!last) { kind = 2; tmap = &tmBb; c0 = tn * (p.BN / 32); }
+                            else if (p.b_nb_last > 0) { kind = 3; tmap = &tmBt; c0 = tn * (p.BN / 32); }
+                            dst_off = kABytes;
+                        } else if (last && p.b_ragged) {
+                            kind = 1;                                   // the partial block after them
+                            dst_off = (uint32_t)kABytes + (uint32_t)p.b_nb_last * 4096u;
+                            c0 = (tn * (p.BN / 32) + p.b_nb_last) * 32;
+                            d1 = kBK;
+                        }
+                    }
                 }
                 const int c2 = is_a ? ab : bb;
-                const CUtensorMap *tmap = is_a ? &tmA : &tmB;
+                // bytes this tile's stages receive (the blocks of the last column tile past N are not fetched)
+                {
+                    const bool last = p.b_mn && p.b_big && tn == p.tiles_n - 1 && (p.b_nb_last != p.BN / 32 || p.b_ragged);
+                    tx = last ? (uint32_t)kABytes + (uint32_t)(p.b_nb_last + (p.b_ragged ? 1 : 0)) * 4096u : p.tx_bytes;
+                }
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
-                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
                     __syncwarp();
-                    if (is_a || is_b)
-                        tma_load_3d(stages + (size_t)stage * p.stage_bytes + dst_off, tmap, &full[stage], c0, c1, c2);
+                    uint8_t *dst = stages + (size_t)stage * p.stage_bytes + dst_off;
+                    if (kind == 1) tma_load_3d(dst, tmap, &full[stage], c0, c1, c2);
+                    else if (kind >= 2) tma_load_4d(dst, tmap, &full[stage], 0, kb * kBK, c0, c2);
                     c0 += d0;
                     c1 += d1;
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
@@ -471,6 +504,26 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
         if (!make_tmap(&tmB, g.B, 3, dims, str, box, p.b_mn ? kTmapSwizzle128Atom32 : kTmapSwizzle128))
             return (int)cudaErrorInvalidValue;
     }
+    // MN-major B through one 4-D box per stage: (32 columns, K, blocks of 32 columns, batch)
+    CUtensorMap tmBb = tmB, tmBt = tmB;
+    p.b_big = 0;
+    if (p.b_mn && g.N >= 32 && p.BN >= 64) {
+        const int per_tile = p.BN / 32, nblk_full = g.N / 32;
+        const int in_last = nblk_full - (p.tiles_n - 1) * per_tile;          // full blocks of the last column tile
+        p.b_nb_last = in_last < 0 ? 0 : (in_last > per_tile ? per_tile : in_last);
+        p.b_ragged = (g.N % 32) != 0 && p.b_nb_last < per_tile;
+        uint64_t dims[4] = {32, (uint64_t)g.K, (uint64_t)nblk_full, p.b_batched ? (uint64_t)g.batch : 1};
+        uint64_t str[3] = {(uint64_t)g.b_ld * 4, 128, p.b_batched ? (uint64_t)g.b_bs * 4 : (uint64_t)g.b_ld * 4 * g.K};
+        uint32_t box[4] = {32, (uint32_t)kBK, (uint32_t)per_tile, 1};
+        bool ok = make_tmap(&tmBb, g.B, 4, dims, str, box, kTmapSwizzle128Atom32);
+        if (ok && p.b_nb_last > 0 && p.b_nb_last < per_tile) {
+            box[2] = (uint32_t)p.b_nb_last;
+            ok = make_tmap(&tmBt, g.B, 4, dims, str, box, kTmapSwizzle128Atom32);
+        } else if (ok) {
+            tmBt = tmBb;
+        }
+        p.b_big = ok ? 1 : 0;
+    }
     if (p.y_tma) {
         uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.M, (uint64_t)g.batch};
         uint64_t str[2] = {(uint64_t)g.y_ld * 4, g.batch > 1 ? (uint64_t)g.y_bs * 4 : (uint64_t)g.y_ld * 4 * g.M};
@@ -486,7 +539,7 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     if (attr_err != cudaSuccess) return (int)attr_err;
     const long long total = (long long)p.tiles_m * p.tiles_n * p.batch;
     const int grid = (int)(total < sms ? total : sms);
-    const cudaError_t le = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB,
+    const cudaError_t le = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB, tmBb, tmBt,
                                       tmY, p);
     count_launch();
     return (int)le;
