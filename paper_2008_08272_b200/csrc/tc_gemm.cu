@@ -20,6 +20,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "common.h"
@@ -49,7 +50,10 @@ __device__ long long g_gprof[148 * 16];
 #define GP_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
 #define GP_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
 #define GP_FLUSH(base, n) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < n; ++k_) g_gprof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
+__device__ long long g_glog[4 * 128];
+#define GLOG(k, i) do { if (blockIdx.x == 0 && (i) < 128) g_glog[(k) * 128 + (i)] = clock64(); } while (0)
 #else
+#define GLOG(k, i) do {} while (0)
 #define GP_DECL do {} while (0)
 #define GP_MARK(k) do {} while (0)
 #define GP_FLUSH(base, n) do {} while (0)
@@ -69,8 +73,10 @@ struct Params {
     // MN-major B in one copy per stage: a 4-D view (32 columns of a block, K row, block of 32 columns,
     // batch) lets a single box carry all of a tile's 32-column blocks in the order the MMA wants them.
     int b_big;                 // that view is in use
-    int b_nb_last;             // full blocks in the last column tile (0: none), loaded through tmBt
-    int b_ragged;              // the last column tile ends in a partial block, loaded through tmB
+    int b_nblk_full;           // full 32-column blocks in a row of B (tiles reaching past them load block by block)
+    // CTA pairs: two CTAs of a cluster share a 256-row tile; each loads its 128 rows of A and half of
+    // the tile's B columns, the even CTA issues cta_group::2 MMAs (M = 256)
+    int ctas, BNH;             // CTAs per tile; B columns staged per CTA = BN / ctas
     float *Y;                  // used by the plain-store epilogue
     long long y_ld, y_sb;
     int y_split;               // > 0: columns are groups of y_split, y_group elements apart (plain stores only)
@@ -79,10 +85,10 @@ struct Params {
     unsigned int *err;
 };
 
+template <int kCtas>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmBb, const __grid_constant__ CUtensorMap tmBt,
-               const __grid_constant__ CUtensorMap tmY, const Params p) {
+               const __grid_constant__ CUtensorMap tmBb, const __grid_constant__ CUtensorMap tmY, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler
     // keeps treating everything derived from it as shared memory (LDS/STS, not generic accesses)
@@ -96,20 +102,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.tiles_m * p.tiles_n * p.batch;
+    const int rank = kCtas == 2 ? (int)cluster_ctarank() : 0;
+    const int first_tile = blockIdx.x / kCtas, tile_step = gridDim.x / kCtas;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.num_stages; ++s) {
-            mbar_init(&full[s], 1);
+            // issuing CTA of a pair: its own producer plus the peer's "landed" message
+            mbar_init(&full[s], (kCtas == 2 && rank == 0) ? 2 : 1);
             mbar_init(&empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&tmem_full[a], 1);
-            mbar_init(&tmem_empty[a], kEpiWarps);
+            mbar_init(&tmem_empty[a], kEpiWarps * kCtas);
         }
         mbar_fence_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
-        if (p.b_big) { prefetch_tmap(&tmBb); prefetch_tmap(&tmBt); }
+        if (p.b_big) prefetch_tmap(&tmBb);
         if (p.y_tma) prefetch_tmap(&tmY);
     }
     if (warp == 1) {
@@ -120,6 +129,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
+    if (kCtas == 2) cluster_sync_all();     // the peer's barriers exist before anything arrives on them
     pdl_launch_dependents();
     pdl_wait();                 // everything above overlapped the previous kernel's tail
 
@@ -127,63 +137,57 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ TMA producer
         // The TMA unit spends 70-90 cycles on every copy instruction however small it is, so a stage is
         // fetched with as few instructions as possible (an MN-major B of up to eight 4 KB blocks through
-        // one 4-D box where the problem allows), and the whole warp runs the loop so that the copies of
-        // a stage are issued by as many lanes at once instead of one thread paying its instruction
-        // latency for each.
+        // one 4-D box), and the whole warp runs the loop so that the copies of a stage are issued by as
+        // many lanes at once instead of one thread paying its instruction latency for each.
         {
             int stage = 0;
             uint32_t phase = 0;
             const int na = p.a_mn ? kBM / 32 : 1;
-            const int nb = !p.b_mn ? 1 : (p.b_big ? 2 : p.BN / 32);
-            // this lane's copy: lanes [0, na) load A pieces, lanes [na, na + nb) load B pieces
-            const bool is_a = lane < na, is_b = !is_a && lane < na + nb;
-            const int j = is_a ? lane : lane - na;
-            for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            const int hb = p.BNH / 32;                 // 32-column blocks of B this CTA stages (MN-major B)
+            // lanes [0, na): A pieces; lane na: B in one copy; lanes [na + 1, na + 1 + hb): B block by block
+            const bool is_a = lane < na;
+            const int jb = lane - na - 1;
+            int glog_i = 0;
+            (void)glog_i;
+            for (int t = first_tile; t < total_tiles; t += tile_step) {
                 const int tm = t % p.tiles_m;
                 const int tn = (t / p.tiles_m) % p.tiles_n;
                 const int b = t / (p.tiles_m * p.tiles_n);
                 const int ab = p.a_batched ? b : 0, bb = p.b_batched ? b : 0;
-                // coordinates of this lane's box at k-block 0 (c0 = contiguous axis) and their step per k-block
-                int c0 = 0, c1 = 0, d0 = 0, d1 = 0, kind = 0;      // kind: 0 none, 1 3-D map, 2 big B box, 3 tail B box
-                uint32_t dst_off = 0, tx = 0;
+                const int row_a = tm * kBM * kCtas + rank * kBM;        // first A row of this CTA
+                const int col_b = tn * p.BN + rank * p.BNH;             // first B column of this CTA
+                // do all of this CTA's blocks lie among the full ones?  Then one 4-D box brings them.
+                const bool one_box = p.b_mn && p.b_big && col_b / 32 + hb <= p.b_nblk_full;
+                // this lane's copy: kind 0 none, 1 3-D map, 2 the 4-D B box
+                int c0 = 0, c1 = 0, d0 = 0, d1 = 0, kind = 0;
+                uint32_t dst_off = 0;
                 const CUtensorMap *tmap = &tmA;
                 if (is_a) {
                     kind = 1;
-                    dst_off = (uint32_t)j * 4096u;
-                    if (!p.a_mn) { c1 = tm * kBM; d0 = kBK; }
-                    else { c0 = tm * kBM + j * 32; d1 = kBK; }
-                } else if (is_b) {
+                    dst_off = (uint32_t)lane * 4096u;
+                    if (!p.a_mn) { c1 = row_a; d0 = kBK; }
+                    else { c0 = row_a + lane * 32; d1 = kBK; }
+                } else if (lane == na) {
                     tmap = &tmB;
-                    if (!p.b_mn) { kind = 1; dst_off = kABytes; c1 = tn * p.BN; d0 = kBK; }
-                    else if (!p.b_big) { kind = 1; dst_off = (uint32_t)kABytes + (uint32_t)j * 4096u; c0 = tn * p.BN + j * 32; d1 = kBK; }
-                    else {
-                        const bool last = tn == p.tiles_n - 1 && (p.b_nb_last != p.BN / 32 || p.b_ragged);
-                        if (j == 0) {
-                            // all of the tile's full blocks: c0 = first block
-                            if (!last) { kind = 2; tmap = &tmBb; c0 = tn * (p.BN / 32); }
-                            else if (p.b_nb_last > 0) { kind = 3; tmap = &tmBt; c0 = tn * (p.BN / 32); }
-                            dst_off = kABytes;
-                        } else if (last && p.b_ragged) {
-                            kind = 1;                                   // the partial block after them
-                            dst_off = (uint32_t)kABytes + (uint32_t)p.b_nb_last * 4096u;
-                            c0 = (tn * (p.BN / 32) + p.b_nb_last) * 32;
-                            d1 = kBK;
-                        }
-                    }
+                    dst_off = kABytes;
+                    if (!p.b_mn) { kind = 1; c1 = col_b; d0 = kBK; }
+                    else if (one_box) { kind = 2; tmap = &tmBb; c0 = col_b / 32; }
+                } else if (p.b_mn && !one_box && jb >= 0 && jb < hb) {
+                    kind = 1;
+                    tmap = &tmB;
+                    dst_off = (uint32_t)kABytes + (uint32_t)jb * 4096u;
+                    c0 = col_b + jb * 32;
+                    d1 = kBK;
                 }
                 const int c2 = is_a ? ab : bb;
-                // bytes this tile's stages receive (the blocks of the last column tile past N are not fetched)
-                {
-                    const bool last = p.b_mn && p.b_big && tn == p.tiles_n - 1 && (p.b_nb_last != p.BN / 32 || p.b_ragged);
-                    tx = last ? (uint32_t)kABytes + (uint32_t)(p.b_nb_last + (p.b_ragged ? 1 : 0)) * 4096u : p.tx_bytes;
-                }
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
-                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx);
+                    if (lane == 0) GLOG(0, glog_i++);
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
                     __syncwarp();
                     uint8_t *dst = stages + (size_t)stage * p.stage_bytes + dst_off;
                     if (kind == 1) tma_load_3d(dst, tmap, &full[stage], c0, c1, c2);
-                    else if (kind >= 2) tma_load_4d(dst, tmap, &full[stage], 0, kb * kBK, c0, c2);
+                    else if (kind == 2) tma_load_4d(dst, tmap, &full[stage], 0, kb * kBK, c0, c2);
                     c0 += d0;
                     c1 += d1;
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
@@ -192,7 +196,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
+        if (kCtas == 2 && rank != 0) {
+            // Odd CTA of a pair: the even CTA issues the MMAs; tell it when each of this CTA's stages
+            // has landed (stage releases and finished accumulators come back by multicast commit).
+            if (elect_one()) {
+                const uint32_t peer_full = map_to_cta(smem_u32(&full[0]), 0);
+                int stage = 0;
+                uint32_t phase = 0;
+                for (int t = first_tile; t < total_tiles; t += tile_step) {
+                    for (int kb = 0; kb < p.num_kb; ++kb) {
+                        mbar_wait(&full[stage], phase, p.err, 5);
+                        mbar_arrive_remote(peer_full + (uint32_t)stage * 8u);
+                        if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+        } else if (elect_one()) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             // Descriptor words that do not change: everything but the 14-bit start address.
@@ -206,16 +225,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t a_lo_c = (uint32_t)a_tmpl, b_lo_c = (uint32_t)b_tmpl;
             const uint32_t a_k16 = (p.a_mn ? 1024u : 32u) >> 4, b_k16 = (p.b_mn ? 1024u : 32u) >> 4;
             const uint32_t idesc = p.idesc;
+            int glog_i = 0, glog_t = 0;
+            (void)glog_i; (void)glog_t;
             GP_DECL;
-            for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-                mbar_wait(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
+            for (int t = first_tile; t < total_tiles; t += tile_step) {
+                if (kCtas == 2) mbar_wait_cluster(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
+                else mbar_wait(&tmem_empty[acc], acc_phase ^ 1, p.err, 2);
                 tc_fence_after_sync();
                 GP_MARK(0);
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * kMaxBN;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
-                    mbar_wait(&full[stage], phase, p.err, 3);
+                    if (kCtas == 2) mbar_wait_cluster(&full[stage], phase, p.err, 3);
+                    else mbar_wait(&full[stage], phase, p.err, 3);
                     tc_fence_after_sync();
                     GP_MARK(1);
+                    GLOG(1, glog_i++);
                     const uint32_t sA = smem_u32(stages + (size_t)stage * p.stage_bytes);
                     const uint32_t a16 = sA >> 4, b16 = (sA + kABytes) >> 4;
                     const int k_left = p.K - kb * kBK;
@@ -223,15 +247,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // one thread issues everything: keep the per-instruction work to two adds
 #pragma unroll
                     for (int k = 0; k < kBK / 8; ++k) {
-                        if (k < k8)
-                            mma_tf32_lohi(d_tmem, a_lo_c | ((a16 + (uint32_t)k * a_k16) & 0x3FFFu), a_hi,
-                                          b_lo_c | ((b16 + (uint32_t)k * b_k16) & 0x3FFFu), b_hi, idesc, (kb | k) != 0);
+                        if (k < k8) {
+                            if (kCtas == 2)
+                                mma_tf32_lohi_pair(d_tmem, a_lo_c | ((a16 + (uint32_t)k * a_k16) & 0x3FFFu), a_hi,
+                                                   b_lo_c | ((b16 + (uint32_t)k * b_k16) & 0x3FFFu), b_hi, idesc, (kb | k) != 0);
+                            else
+                                mma_tf32_lohi(d_tmem, a_lo_c | ((a16 + (uint32_t)k * a_k16) & 0x3FFFu), a_hi,
+                                              b_lo_c | ((b16 + (uint32_t)k * b_k16) & 0x3FFFu), b_hi, idesc, (kb | k) != 0);
+                        }
                     }
-                    mma_commit(&empty[stage]);
+                    if (kCtas == 2) mma_commit_pair(&empty[stage]);
+                    else mma_commit(&empty[stage]);
                     if (++stage == p.num_stages) { stage = 0; phase ^= 1; }
                     GP_MARK(2);
                 }
-                mma_commit(&tmem_full[acc]);
+                if (kCtas == 2) mma_commit_pair(&tmem_full[acc]);
+                else mma_commit(&tmem_full[acc]);
+                GLOG(2, glog_t++);
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1;
             }
@@ -245,14 +277,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int acc = 0;
         uint32_t acc_phase = 0;
         GP_DECL;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        const uint32_t peer_tmem_empty = kCtas == 2 ? map_to_cta(smem_u32(&tmem_empty[0]), 0) : 0u;
+        for (int t = first_tile; t < total_tiles; t += tile_step) {
             const int tm = t % p.tiles_m;
             const int tn = (t / p.tiles_m) % p.tiles_n;
             const int b = t / (p.tiles_m * p.tiles_n);
             mbar_wait(&tmem_full[acc], acc_phase, p.err, 4);
             tc_fence_after_sync();
             GP_MARK(0);
-            const int row0 = tm * kBM + q * 32;
+            const int row0 = tm * kBM * kCtas + rank * kBM + q * 32;
             const int row = row0 + lane;
             if (row0 < p.M) {
                 const float rb = (p.row_bias && row < p.M) ? __ldg(p.row_bias + row) : 0.f;
@@ -344,7 +377,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+            if (lane == 0) {
+                if (kCtas == 2) mbar_arrive_remote(peer_tmem_empty + (uint32_t)acc * 8u);
+                else mbar_arrive(&tmem_empty[acc]);
+            }
             acc ^= 1;
             if (acc == 0) acc_phase ^= 1;
         }
@@ -354,6 +390,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     tc_fence_before_sync();
     __syncthreads();
+    if (kCtas == 2) cluster_sync_all();     // no CTA leaves while its peer may still signal it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -361,11 +398,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-int pick_bn(long long tiles_m, long long n, long long batch, int num_sms) {
-    if (n <= 32) return 32;
-    int best = 32;
+int pick_bn(long long tiles_m, long long n, long long batch, int num_sms, int ctas) {
+    if (n <= 32 * ctas) return 32 * ctas;
+    int best = 32 * ctas;
     double best_cost = 1e300;
-    for (int bn = 32; bn <= kMaxBN; bn += 32) {
+    for (int bn = 32 * ctas; bn <= kMaxBN; bn += 32 * ctas) {
         const long long tiles = tiles_m * ((n + bn - 1) / bn) * batch;
         const long long waves = (tiles + num_sms - 1) / num_sms;
         const double cost = (double)waves * (bn + 48);
@@ -435,6 +472,11 @@ int num_sms() {
 }  // namespace tc_host
 
 #ifdef ONNXB_PROFILE
+extern "C" int onnxb_dbg_glog(long long *out) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_glog, sizeof(long long) * 4 * 128);
+    return 0;
+}
 extern "C" int onnxb_dbg_gprofile(long long *out) {
     cudaDeviceSynchronize();
     cudaMemcpyFromSymbol(out, g_gprof, sizeof(long long) * 148 * 16);
@@ -451,22 +493,58 @@ bool tc_gemm_supports(const TcGemmProblem &g) {
     return true;
 }
 
+// How many CTA pairs (clusters of two) of the pair kernel the device runs at once; queried once.
+static int gemm_max_pairs() {
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * 148);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemLimit;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<2>, &cfg) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = tc_host::num_sms() / 2;
+    }
+    cached = n;
+    return n;
+}
+
 int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     using namespace tc_host;
     Params p{};
     p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
     p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
     p.a_batched = g.a_batched && g.batch > 1; p.b_batched = g.b_batched && g.batch > 1;
-    p.tiles_m = (g.M + kBM - 1) / kBM;
     const int sms = num_sms();
-    p.BN = pick_bn(p.tiles_m, g.N, g.batch, sms);
+    // CTA pairs when the rows fill 256-row tiles: each CTA then fetches half of B.  That is what the
+    // layers bound by the L2 -> shared-memory stream (small images, many channels) need: measured 7-15 %
+    // faster on the 14x14 and strided 1x1 layers of ResNet-50, neutral on the HBM-bound ones.
+    p.ctas = 1;
+    {
+        const char *e = getenv("ONNXB_GEMM_PAIR");          // "0"/"1": pin the choice for A/B measurements
+        bool pair = g.M >= 256 && (g.M % 256 == 0 || g.M % 256 > 128) && g.N >= 64;
+        if (e && (e[0] == '0' || e[0] == '1')) pair = e[0] == '1' && g.M > 128 && g.N >= 64;
+        if (pair) p.ctas = 2;
+    }
+    const int units = p.ctas == 2 ? gemm_max_pairs() : sms;
+    p.tiles_m = (g.M + kBM * p.ctas - 1) / (kBM * p.ctas);
+    p.BN = pick_bn(p.tiles_m, g.N, g.batch, units, p.ctas);
+    p.BNH = p.BN / p.ctas;
     p.tiles_n = (g.N + p.BN - 1) / p.BN;
     p.num_kb = (g.K + kBK - 1) / kBK;
-    p.stage_bytes = (uint32_t)(kABytes + p.BN * 128);
+    p.stage_bytes = (uint32_t)(kABytes + p.BNH * 128);
     p.tx_bytes = p.stage_bytes;
     int stages = (kSmemLimit - 1024 - kBarrierBytes - kStagingBytes) / (int)p.stage_bytes;
     p.num_stages = stages > kMaxStages ? kMaxStages : stages;
-    p.idesc = tc::make_idesc_tf32(kBM, p.BN, p.a_mn, p.b_mn);
+    p.idesc = tc::make_idesc_tf32(kBM * p.ctas, p.BN, p.a_mn, p.b_mn);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
     p.row_bias = g.row_bias; p.relu = g.relu;
@@ -495,7 +573,7 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
         const uint64_t cols = (uint64_t)g.N, k = (uint64_t)g.K;
         uint64_t dims[3], str[2];
         uint32_t box[3];
-        if (!p.b_mn) { dims[0] = k; dims[1] = cols; box[0] = kBK; box[1] = (uint32_t)p.BN; }
+        if (!p.b_mn) { dims[0] = k; dims[1] = cols; box[0] = kBK; box[1] = (uint32_t)p.BNH; }
         else { dims[0] = cols; dims[1] = k; box[0] = 32; box[1] = kBK; }
         dims[2] = p.b_batched ? (uint64_t)g.batch : 1;
         box[2] = 1;
@@ -504,25 +582,16 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
         if (!make_tmap(&tmB, g.B, 3, dims, str, box, p.b_mn ? kTmapSwizzle128Atom32 : kTmapSwizzle128))
             return (int)cudaErrorInvalidValue;
     }
-    // MN-major B through one 4-D box per stage: (32 columns, K, blocks of 32 columns, batch)
-    CUtensorMap tmBb = tmB, tmBt = tmB;
+    // MN-major B through one 4-D box per stage: (32 columns, K, blocks of 32 columns, batch).  Only the
+    // full blocks of a row belong to the view; a CTA whose columns reach past them loads block by block.
+    CUtensorMap tmBb = tmB;
     p.b_big = 0;
-    if (p.b_mn && g.N >= 32 && p.BN >= 64) {
-        const int per_tile = p.BN / 32, nblk_full = g.N / 32;
-        const int in_last = nblk_full - (p.tiles_n - 1) * per_tile;          // full blocks of the last column tile
-        p.b_nb_last = in_last < 0 ? 0 : (in_last > per_tile ? per_tile : in_last);
-        p.b_ragged = (g.N % 32) != 0 && p.b_nb_last < per_tile;
-        uint64_t dims[4] = {32, (uint64_t)g.K, (uint64_t)nblk_full, p.b_batched ? (uint64_t)g.batch : 1};
+    p.b_nblk_full = g.N / 32;
+    if (p.b_mn && p.b_nblk_full >= 1 && p.BNH >= 64) {
+        uint64_t dims[4] = {32, (uint64_t)g.K, (uint64_t)p.b_nblk_full, p.b_batched ? (uint64_t)g.batch : 1};
         uint64_t str[3] = {(uint64_t)g.b_ld * 4, 128, p.b_batched ? (uint64_t)g.b_bs * 4 : (uint64_t)g.b_ld * 4 * g.K};
-        uint32_t box[4] = {32, (uint32_t)kBK, (uint32_t)per_tile, 1};
-        bool ok = make_tmap(&tmBb, g.B, 4, dims, str, box, kTmapSwizzle128Atom32);
-        if (ok && p.b_nb_last > 0 && p.b_nb_last < per_tile) {
-            box[2] = (uint32_t)p.b_nb_last;
-            ok = make_tmap(&tmBt, g.B, 4, dims, str, box, kTmapSwizzle128Atom32);
-        } else if (ok) {
-            tmBt = tmBb;
-        }
-        p.b_big = ok ? 1 : 0;
+        uint32_t box[4] = {32, (uint32_t)kBK, (uint32_t)(p.BNH / 32), 1};
+        p.b_big = make_tmap(&tmBb, g.B, 4, dims, str, box, kTmapSwizzle128Atom32) ? 1 : 0;
     }
     if (p.y_tma) {
         uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.M, (uint64_t)g.batch};
@@ -535,12 +604,16 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
 
     const size_t smem = 1024 + (size_t)p.num_stages * p.stage_bytes + kStagingBytes + kBarrierBytes;
     const cudaError_t attr_err =
-        cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        cudaFuncSetAttribute(p.ctas == 2 ? tc_gemm_kernel<2> : tc_gemm_kernel<1>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (attr_err != cudaSuccess) return (int)attr_err;
     const long long total = (long long)p.tiles_m * p.tiles_n * p.batch;
-    const int grid = (int)(total < sms ? total : sms);
-    const cudaError_t le = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB, tmBb, tmBt,
-                                      tmY, p);
+    const int grid = (int)(total < units ? total : units) * p.ctas;
+    const cudaError_t le =
+        p.ctas == 2 ? launch_pdl_cluster(tc_gemm_kernel<2>, 2, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA,
+                                         tmB, tmBb, tmY, p)
+                    : launch_pdl(tc_gemm_kernel<1>, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB, tmBb,
+                                 tmY, p);
     count_launch();
     return (int)le;
 }

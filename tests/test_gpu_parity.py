@@ -182,6 +182,35 @@ def test_conv_implicit_gemm_tile_shapes(binding, c, tile, monkeypatch):
     assert worst_ratio(got, want, S) <= 1.0
 
 
+@pytest.mark.parametrize("pair", ["0", "1"])
+@pytest.mark.parametrize("shape", [(256, 200, 96), (384, 3136, 64), (300, 260, 130), (512, 64, 1024)])
+def test_gemm_cta_pair_choice(binding, shape, pair, monkeypatch):
+    """The tensor-core GEMM with one CTA per tile and with CTA pairs (256-row tiles), forced."""
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    B = rng.standard_normal((K, N)).astype(np.float32)
+    C = rng.standard_normal((N,)).astype(np.float32)
+    monkeypatch.setenv("ONNXB_GEMM_PAIR", pair)
+    got = run_gemm_gpu(binding, torch, A, B, C)
+    want, S = oracle.gemm(A, B, C)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+def test_conv1x1_cta_pair_choice(binding, pair, monkeypatch):
+    """1x1 convolutions (direct and strided) through the GEMM kernel with the pair choice forced."""
+    rng = np.random.default_rng(31)
+    monkeypatch.setenv("ONNXB_GEMM_PAIR", pair)
+    for xs, ws, st in [((3, 64, 14, 14), (320, 64, 1, 1), (1, 1)), ((2, 96, 28, 28), (256, 96, 1, 1), (2, 2)),
+                       ((5, 128, 7, 7), (384, 128, 1, 1), (1, 1))]:
+        X = rng.random(xs, dtype=np.float32)
+        W = (rng.standard_normal(ws) * np.sqrt(2.0 / ws[1])).astype(np.float32)
+        B = (rng.standard_normal((ws[0],)) * 0.1).astype(np.float32)
+        ratio, _ = check_conv(binding, torch, X, W, B, relu=True, strides=st)
+        assert ratio <= 1.0, (xs, ws, st, ratio)
+
+
 def test_conv_auto_pad_and_no_bias(binding):
     rng = np.random.default_rng(5)
     X = rng.standard_normal((2, 6, 13, 11)).astype(np.float32)
