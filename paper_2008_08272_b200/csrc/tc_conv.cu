@@ -393,10 +393,26 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         uint32_t rphase = 0, aphase = 0, tile_it = 0;
         PROF_DECL;
         const uint32_t a_full_addr = kCtas == 2 ? map_to_cta(smem_u32(&bars->a_full[0]), 0) : 0u;
+        // What does not depend on the tile is worked out once: where a unit's operand row goes, and
+        // which slot of which parity plane it reads.
+        uint32_t udst[kOwned];                     // byte offset of the unit's operand row inside an A stage | chunk index
+        uint32_t ujp[kOwned];                      // slot within the plane | plane << 28
+#pragma unroll
+        for (int i = 0; i < kOwned; ++i) {
+            udst[i] = 0;
+            ujp[i] = 0;
+            if (i < nu) {
+                const int u = xt + i * kXformThreads;
+                const int ch = conv_fdiv(u, g.planes * g.SLOTS, g.dv_pss), idx = u - ch * per_stage_slots;
+                // operand rows are 16 bytes apart: the low four bits carry the unit's chunk index
+                udst[i] = ((uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u) | (uint32_t)ch;
+                const int pl = conv_fdiv(idx, g.SLOTS, g.dv_SLOTS), j = idx - pl * g.SLOTS;
+                ujp[i] = (uint32_t)j | ((uint32_t)pl << 28);
+            }
+        }
         for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
             const long long G0 = ((t / cgt) * kCtas + rank) * tile_rows;
             int uoff[kOwned];                      // raw float offset of the unit's first channel, -1 = padding
-            uint32_t udst[kOwned];                 // byte offset of the unit's operand row inside an A stage
             const int rot = cb_rotation(t, ncb);
             {
                 // per-thread offsets of the tile, from its segment table (ready before the data)
@@ -408,14 +424,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
 #pragma unroll
                 for (int i = 0; i < kOwned; ++i) {
                     uoff[i] = -1;
-                    udst[i] = 0;
                     if (i < nu) {
-                        const int u = xt + i * kXformThreads;
-                        const int ch = conv_fdiv(u, g.planes * g.SLOTS, g.dv_pss), idx = u - ch * per_stage_slots;
-                        // operand rows are 16 bytes apart: the low four bits carry the unit's chunk index
-                        udst[i] = ((uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u) | (uint32_t)ch;
-                        const int pl = conv_fdiv(idx, g.SLOTS, g.dv_SLOTS), j = idx - pl * g.SLOTS;
-                        const uint32_t Gs = (uint32_t)G0 + (uint32_t)j;     // the planner keeps slots below 2^31
+                        const int ch = (int)(udst[i] & 15u), pl = (int)(ujp[i] >> 28);
+                        const uint32_t Gs = (uint32_t)G0 + (ujp[i] & 0x0FFFFFFFu);     // the planner keeps slots below 2^31
                         if (Gs < (uint32_t)g.total_slots) {
                             const int n = conv_fdiv((int)Gs, g.L, g.dv_L);
                             const int uu = (int)Gs - n * g.L;
@@ -455,28 +466,33 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 uint8_t *adst = a_st + (size_t)as * g.a_stage_bytes;
                 const int cbx = cb + rot < ncb ? cb + rot : cb + rot - ncb;
                 const int c_left = g.Cg - cbx * KB;    // channels of this block that exist
-                {
-                    // all reads first (independent, so their latencies overlap), then round and store;
-                    // channels past the end of the group (last block only) read as zero
-                    float v[kOwned][4];
+                // In two batches of five units: all reads of a batch first (independent, so their latencies
+                // overlap), then round and store; channels past the end of the group (last block only)
+                // read as zero.
 #pragma unroll
-                    for (int i = 0; i < kOwned; ++i) {
-                        v[i][0] = v[i][1] = v[i][2] = v[i][3] = 0.f;
+                for (int h0 = 0; h0 < kOwned; h0 += kOwned / 2) {
+                    float v[kOwned / 2][4];
+#pragma unroll
+                    for (int k = 0; k < kOwned / 2; ++k) {
+                        const int i = h0 + k;
+                        v[k][0] = v[k][1] = v[k][2] = v[k][3] = 0.f;
                         if (i < nu && uoff[i] >= 0) {
                             const float *r = raw + uoff[i];
                             const int left = c_left - (int)(udst[i] & 15u) * 4;
-                            if (left > 0) v[i][0] = r[0];
-                            if (left > 1) v[i][1] = r[cp];
-                            if (left > 2) v[i][2] = r[2 * cp];
-                            if (left > 3) v[i][3] = r[3 * cp];
+                            if (left > 0) v[k][0] = r[0];
+                            if (left > 1) v[k][1] = r[cp];
+                            if (left > 2) v[k][2] = r[2 * cp];
+                            if (left > 3) v[k][3] = r[3 * cp];
                         }
                     }
 #pragma unroll
-                    for (int i = 0; i < kOwned; ++i)
+                    for (int k = 0; k < kOwned / 2; ++k) {
+                        const int i = h0 + k;
                         if (i < nu)
                             *reinterpret_cast<float4 *>(adst + (udst[i] & ~15u)) =
-                                make_float4(round_tf32(v[i][0]), round_tf32(v[i][1]), round_tf32(v[i][2]),
-                                            round_tf32(v[i][3]));
+                                make_float4(round_tf32(v[k][0]), round_tf32(v[k][1]), round_tf32(v[k][2]),
+                                            round_tf32(v[k][3]));
+                    }
                 }
                 PROF_MARK(2);
                 fence_proxy_async_smem();
