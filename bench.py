@@ -432,6 +432,37 @@ def run_ours(args):
     return 0
 
 
+def run_probe_tf32():
+    """TF32 tcgen05.mma issue-rate ceiling (operands resident in shared memory, every SM busy): one JSON line."""
+    import torch
+    from paper_2008_08272_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    binding.load(build_if_missing=False)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    max_mhz = measured_clock_max_mhz()
+    out = {"probe": "tcgen05.mma kind::tf32, 128 x N x 8, operands resident in shared memory", "sms": sms,
+           "sm_max_mhz": max_mhz, "shapes": {}}
+    for n in (64, 128, 256):
+        cyc = min(binding.probe_tf32_mma_rate(n, 4096) for _ in range(3))
+        mac = 128.0 * n * 8 / cyc
+        out["shapes"][str(n)] = {"cycles_per_instruction": round(cyc, 2), "ideal": n // 2,
+                                 "mac_per_clk_per_sm": round(mac, 1),
+                                 "tflops_at_max_clock": round(2 * mac * sms * max_mhz * 1e6 / 1e12, 1)}
+    print(json.dumps(out))
+    return 0
+
+
+def measured_clock_max_mhz():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh).get("sm_max_mhz", 1965.0))
+    except (OSError, ValueError):
+        return 1965.0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -441,10 +472,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: run only the convolutions whose name contains this")
     ap.add_argument("--batch", type=int, default=64, help="images per convolution (the benchmark proper uses 64)")
+    ap.add_argument("--probe-tf32", action="store_true",
+                    help="measure the issue-rate ceiling of the TF32 tensor-core instruction instead of the step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         return run_reference(args)
+    if args.probe_tf32:
+        return run_probe_tf32()
     return run_ours(args)
 
 

@@ -218,6 +218,19 @@ void onnxb_set_kernel_override(int family);
 /* Number of kernels this library has launched since it was loaded (all streams). */
 uint64_t onnxb_launch_count(void);
 
+/*
+ * Measurement aid (no operator of the paper behind it; Sec. 4.2 reports whole-model times only):
+ * the issue-rate ceiling of the TF32 tensor-core instruction the Conv and Gemm kernels are built
+ * from.  Every SM issues `instructions` tcgen05.mma kind::tf32 instructions of shape 128 x n x 8
+ * back to back on operands already in shared memory; *cycles_per_instruction receives the SM
+ * cycles per instruction of the slowest SM (ideal: n / 2).  n: multiple of 16 in [16, 256];
+ * instructions in [16, 2^20].  Unlike the run calls this one allocates a small device buffer,
+ * launches on `cuda_stream` and synchronises it before returning.  Host pointer out; ERR_ATTR for
+ * arguments out of range, ERR_CUDA if the device refuses.
+ */
+onnxb_status onnxb_probe_tf32_mma_rate(int n, int instructions, double *cycles_per_instruction,
+                                       void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

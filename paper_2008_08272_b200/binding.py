@@ -24,6 +24,7 @@ EXPORTS = [
     "onnx_conv2d_desc_destroy", "onnx_conv2d_run_static", "onnx_conv2d_static_scratch_bytes",
     "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
+    "onnxb_probe_tf32_mma_rate",
 ]
 
 
@@ -90,6 +91,8 @@ def load(build_if_missing: bool = True):
     lib.onnxb_set_kernel_override.argtypes = [ctypes.c_int]
     lib.onnxb_launch_count.restype = ctypes.c_uint64
     lib.onnxb_launch_count.argtypes = []
+    lib.onnxb_probe_tf32_mma_rate.restype = ctypes.c_int
+    lib.onnxb_probe_tf32_mma_rate.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double), vp]
     _lib = lib
     return lib
 
@@ -253,3 +256,12 @@ def set_kernel_override(family) -> None:
 
 def launch_count() -> int:
     return int(load().onnxb_launch_count())
+
+
+def probe_tf32_mma_rate(n: int, instructions: int = 4096, stream=None) -> float:
+    """``onnxb_probe_tf32_mma_rate``: SM cycles per 128 x n x 8 TF32 MMA with operands resident
+    in shared memory (the tensor pipe's ceiling for that shape; ideal n / 2)."""
+    out = ctypes.c_double()
+    _check(load().onnxb_probe_tf32_mma_rate(int(n), int(instructions), ctypes.byref(out), _stream_ptr(stream)),
+           "onnxb_probe_tf32_mma_rate")
+    return float(out.value)

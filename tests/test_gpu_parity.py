@@ -347,6 +347,17 @@ def test_sweep_index_mapping_on_full_batch(binding):
             assert np.array_equal(got[:, m], want), (C, HW, m)
 
 
+def test_tf32_mma_rate_probe(binding):
+    """The measurement aid returns a plausible figure: never faster than the tensor pipe's ideal
+    n/2 cycles per 128 x n x 8 instruction, and within a factor two of it; bad arguments are refused."""
+    for n in (64, 256):
+        cyc = binding.probe_tf32_mma_rate(n, 1024)
+        assert n / 2 * 0.98 <= cyc <= n, (n, cyc)
+    with pytest.raises(binding.OnnxB200Error):
+        binding.probe_tf32_mma_rate(100, 1024)
+    assert binding.last_device_status() == 0
+
+
 def test_run_rejects_short_workspace_and_host_tensors(binding):
     x = torch.zeros((1, 4, 8, 8), device="cuda")
     w = torch.zeros((4, 4, 3, 3), device="cuda")
