@@ -167,23 +167,25 @@ __device__ __forceinline__ float gather_round(float v) {
 
 __global__ void __launch_bounds__(256)
 gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, unsigned total, unsigned pitch, unsigned NPQ,
-                 unsigned PQ, unsigned Q, unsigned C, unsigned HW, unsigned rowstep, unsigned sw, int merged) {
+                 unsigned PQ, unsigned Q, unsigned C, unsigned HW, unsigned rowstep, unsigned sw, int merged,
+                 const ConvDivisor dv_pitch, const ConvDivisor dv_PQ, const ConvDivisor dv_Q) {
     tc::pdl_launch_dependents();
+    // the three divisions per element are multiply-and-shift by constants the host prepares
     for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < total; i += gridDim.x * 256u) {
-        const unsigned row = i / pitch;               // merged: channel; per image: n*C + c
+        const unsigned row = (unsigned)conv_fdiv((int)i, (int)pitch, dv_pitch);   // merged: channel; per image: n*C + c
         const unsigned j = i - row * pitch;
         float v = 0.f;
         if (j < NPQ) {
             unsigned plane, r;
             if (merged) {
-                const unsigned n = j / PQ;
+                const unsigned n = (unsigned)conv_fdiv((int)j, (int)PQ, dv_PQ);
                 r = j - n * PQ;
                 plane = n * C + row;
             } else {
                 r = j;
                 plane = row;
             }
-            const unsigned p = r / Q, q = r - p * Q;
+            const unsigned p = (unsigned)conv_fdiv((int)r, (int)Q, dv_Q), q = r - p * Q;
             v = gather_round(__ldg(X + (size_t)plane * HW + p * rowstep + q * sw));
         }
         Xg[i] = v;
@@ -361,11 +363,12 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
                                                            reinterpret_cast<float4 *>(Xg), (unsigned)total4, PQ4, Q4,
                                                            HW4, rowstep4);
     } else {
-        const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, 148LL * 32);
+        const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, 148LL * 64);
         gather1x1_kernel<<<blocks, 256, 0, st>>>(X, Xg, (unsigned)total, (unsigned)pitch,
                                                  (unsigned)(merged ? g.N * g.P * g.Q : g.P * g.Q), (unsigned)(g.P * g.Q),
                                                  (unsigned)g.Q, (unsigned)g.C, (unsigned)(g.H * g.W),
-                                                 (unsigned)(g.sh * g.W), (unsigned)g.sw, merged ? 1 : 0);
+                                                 (unsigned)(g.sh * g.W), (unsigned)g.sw, merged ? 1 : 0,
+                                                 conv_divisor((int)pitch), conv_divisor(g.P * g.Q), conv_divisor(g.Q));
     }
     count_launch();
     return (int)cudaGetLastError();
