@@ -212,6 +212,23 @@ def run_reference(args):
     return 0
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """The slowest rank's figure (every rank gets it): the replicas run independently, so the job's
+    step time is the maximum of theirs.  Uses the default process group (NCCL on GPUs, gloo on CPU)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tflops(world: int, flops_per_replica_step: float, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas that each do one step in ms_per_step."""
+    return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -295,12 +312,9 @@ def run_ours(args):
     launches = binding.launch_count() - launches0
     ms_total = t_start.elapsed_time(t_end)
     assert binding.last_device_status() == 0, "a device-side wait timed out"
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
-    value = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+    value = job_tflops(world, flops_per_step, ms_per_step)
 
     # Per-op durations: the same K steps again, now with an event after every op.  (Events between
     # kernels forbid the early start of the next kernel that back-to-back launches get, so this pass is
@@ -380,11 +394,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * flops_per_step / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+    e2e_value = job_tflops(world, flops_per_step, e2e_ms)
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, single GPU runs only)
     cpu = None
