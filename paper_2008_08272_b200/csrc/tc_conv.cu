@@ -46,6 +46,7 @@ constexpr int kXformThreads = kXformWarps * 32;
 constexpr int kEpiWarps = 8;
 constexpr int kOwned = 10;                 // (slot, chunk) units of an A stage one transform thread may own
 constexpr int kMaxRawStages = 4;
+constexpr int kMaxAStages = 3;
 constexpr int kMaxSpb = 8;                 // K-steps per weight stage (the MMA issue loop is unrolled over them)
 constexpr int kMaxBStages = 12;
 constexpr int kSmemLimit = 232448;
@@ -54,7 +55,7 @@ constexpr int kSegBytes = 256;             // >= sizeof(TcConvSegs)
 static_assert(sizeof(TcConvSegs) <= kSegBytes, "segment table does not fit its slot");
 
 struct Bars {
-    uint64_t raw_full[kMaxRawStages], raw_empty[kMaxRawStages], a_full[2], a_empty[2];
+    uint64_t raw_full[kMaxRawStages], raw_empty[kMaxRawStages], a_full[kMaxAStages], a_empty[kMaxAStages];
     uint64_t b_full[kMaxBStages], b_empty[kMaxBStages];
     uint64_t acc_full[2], acc_empty[2];
     uint64_t seg_full[2], seg_empty[2];      // segment tables, one per tile parity
@@ -145,7 +146,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     // keeps treating everything derived from it as shared memory (LDS/STS, not generic accesses)
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *a_st = smem;
-    uint8_t *raw_st = a_st + 2 * (size_t)g.a_stage_bytes;
+    uint8_t *raw_st = a_st + (size_t)g.na_stages * g.a_stage_bytes;
     uint8_t *b_st = raw_st + (size_t)g.nr_stages * g.raw_stage_bytes;
     uint8_t *seg_st = b_st + (size_t)g.nb_stages * g.b_stage_bytes;
     Bars *bars = reinterpret_cast<Bars *>(seg_st + kMaxRawStages * kSegBytes);
@@ -165,7 +166,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             mbar_init(&bars->raw_full[s], 1);
             mbar_init(&bars->raw_empty[s], kXformWarps);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < g.na_stages; ++s) {
             mbar_init(&bars->a_full[s], kXformWarps * kCtas);      // waited on by the issuing CTA only
             mbar_init(&bars->a_empty[s], 1);
         }
@@ -369,8 +370,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                     if (kCtas == 2) mma_commit_pair(&bars->a_empty[as]);
                     else mma_commit(&bars->a_empty[as]);
                     LOG(4, cb);
-                    as ^= 1;
-                    if (as == 0) aphase ^= 1;
+                    if (++as == g.na_stages) { as = 0; aphase ^= 1; }
                 }
                 if (kCtas == 2) mma_commit_pair(&bars->acc_full[ab]);
                 else mma_commit(&bars->acc_full[ab]);
@@ -505,8 +505,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 PROF_MARK(3);
                 if (xt == 0) LOG(7, cb);
                 if (++rs == nr) { rs = 0; rphase ^= 1; }
-                as ^= 1;
-                if (as == 0) aphase ^= 1;
+                if (++as == g.na_stages) { as = 0; aphase ^= 1; }
             }
 
         }
@@ -775,10 +774,22 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
     }
     // Raw stages: a third one (the raw tiles come from L2/HBM with a microsecond of latency) when that
     // still leaves 64 KB for the weight ring.
-    const long long base_fixed = 1024 + 2LL * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
+    g.na_stages = 2;
     g.nr_stages = 2;
-    for (int nr = 3; nr <= kMaxRawStages - 1; ++nr)
-        if (kSmemLimit - base_fixed - (long long)nr * g.raw_stage_bytes >= 65536) g.nr_stages = nr;
+    {
+        // "ONNXB_CONV_STAGES=a,r" pins the operand / raw stage counts for A/B measurements
+        int fa = 0, fr = 0;
+        const char *e = getenv("ONNXB_CONV_STAGES");
+        if (e && sscanf(e, "%d,%d", &fa, &fr) == 2 && fa >= 2 && fa <= kMaxAStages && fr >= 2 && fr < kMaxRawStages) {
+            g.na_stages = fa;
+            g.nr_stages = fr;
+        } else {
+            const long long bf = 1024 + 2LL * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
+            for (int nr = 3; nr <= kMaxRawStages - 1; ++nr)
+                if (kSmemLimit - bf - (long long)nr * g.raw_stage_bytes >= 65536) g.nr_stages = nr;
+        }
+    }
+    const long long base_fixed = 1024 + (long long)g.na_stages * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
     const long long fixed = base_fixed + (long long)g.nr_stages * g.raw_stage_bytes;
     const long long room = kSmemLimit - fixed;
     while (room < 3LL * g.spb * g.b_step_bytes && g.spb > 1) g.spb = (g.spb + 1) / 2;   // keep three stages in flight
@@ -944,7 +955,7 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     } else {
         memset(&tmX, 0, sizeof tmX);
     }
-    const size_t smem = 1024 + 2 * (size_t)plan.a_stage_bytes + (size_t)plan.nr_stages * plan.raw_stage_bytes +
+    const size_t smem = 1024 + (size_t)plan.na_stages * plan.a_stage_bytes + (size_t)plan.nr_stages * plan.raw_stage_bytes +
                         (size_t)plan.nb_stages * plan.b_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
     const bool pair = plan.ctas == 2;
     cudaError_t e = cudaFuncSetAttribute(pair ? tc_conv_kernel<2> : tc_conv_kernel<1>,

@@ -60,7 +60,7 @@ struct TcConvPlan {
     int raw_mode;                    // 0: tensor-map boxes [KB][BOXP] over X seen as (H*W, N*C); 1: whole-image slabs
     int BOXP;
     // shared memory carve-up (bytes)
-    int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages, nr_stages;
+    int a_stage_bytes, raw_stage_bytes, b_stage_bytes, nb_stages, nr_stages, na_stages;
     int spb, b_step_bytes, b_steps;  // K-steps per weight stage, bytes of one step's weights, weight stages per block
     int chunk_pitch, plane_pitch;    // bytes between 4-channel chunks / parity planes inside an A stage
     uint32_t idesc;
