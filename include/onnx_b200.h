@@ -194,6 +194,20 @@ onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float beta,
                            int fuse_relu, float *Y, void *workspace, size_t workspace_bytes,
                            void *cuda_stream);
 
+/*
+ * onnx_matmul_add_run - the pair MatMul(A, B) followed by Add(., C) that the compiler's
+ * graph rewriting fuses into one Gemm (Sec. 3.4.3, the MulAddToGemm pattern):
+ *
+ *   Y[i,j] = relu?( sum_k A[i,k] * B[k,j] + Cb[i,j] )
+ *
+ * A [M,K], B [K,N], C broadcast as in onnx_gemm_run (C == NULL: plain MatMul), Y [M,N];
+ * exactly onnx_gemm_run with transA = transB = 0 and alpha = beta = 1, same pointers,
+ * workspace and errors.
+ */
+onnxb_status onnx_matmul_add_run(int64_t M, int64_t N, int64_t K, const float *A, const float *B,
+                                 const float *C, int c_rank, const int64_t *c_dims, int fuse_relu,
+                                 float *Y, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char *onnxb_status_string(onnxb_status status);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "onnx_conv2d_desc_destroy", "onnx_conv2d_run_static", "onnx_conv2d_static_scratch_bytes",
     "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
-    "onnxb_probe_tf32_mma_rate",
+    "onnxb_probe_tf32_mma_rate", "onnx_matmul_add_run",
 ]
 
 
@@ -83,6 +83,9 @@ def load(build_if_missing: bool = True):
     lib.onnx_gemm_run.restype = ctypes.c_int
     lib.onnx_gemm_run.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_float, i64, i64, i64,
                                   vp, vp, vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.c_int, vp, vp, sz, vp]
+    lib.onnx_matmul_add_run.restype = ctypes.c_int
+    lib.onnx_matmul_add_run.argtypes = [i64, i64, i64, vp, vp, vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.c_int, vp,
+                                        vp, sz, vp]
     lib.onnxb_status_string.restype = ctypes.c_char_p
     lib.onnxb_status_string.argtypes = [ctypes.c_int]
     lib.onnxb_last_device_status.restype = ctypes.c_int
@@ -265,3 +268,28 @@ def probe_tf32_mma_rate(n: int, instructions: int = 4096, stream=None) -> float:
     _check(load().onnxb_probe_tf32_mma_rate(int(n), int(instructions), ctypes.byref(out), _stream_ptr(stream)),
            "onnxb_probe_tf32_mma_rate")
     return float(out.value)
+
+
+def onnx_matmul_add(A, B, C=None, *, fuse_relu=False, Y=None, workspace=None, stream=None):
+    """``onnx_matmul_add_run``: Y = relu?(A @ B + C), the MatMul + Add pair as one fused Gemm."""
+    import torch
+    lib = load()
+    M, K = A.shape
+    if B.shape[0] != K:
+        raise OnnxB200Error(3, "onnx_matmul_add: inner dimensions differ")
+    N = B.shape[1]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    c_rank, c_dims = 0, None
+    if C is not None:
+        c_rank = C.dim()
+        c_dims = (ctypes.c_int64 * max(c_rank, 1))(*[int(v) for v in C.shape])
+    need = gemm_workspace_bytes(False, False, M, N, K)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=A.device)
+    ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    ws_len = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib.onnx_matmul_add_run(M, N, K, _dev_ptr(A, "A"), _dev_ptr(B, "B"), _dev_ptr(C, "C", allow_none=True),
+                                   c_rank, c_dims, int(bool(fuse_relu)), _dev_ptr(Y, "Y"), ws_ptr, ws_len,
+                                   _stream_ptr(stream)), "onnx_matmul_add_run")
+    return Y

@@ -198,3 +198,12 @@ extern "C" onnxb_status onnxb_last_device_status(void *cuda_stream) {
     }
     return ONNXB_OK;
 }
+
+// MatMul followed by Add, as the graph rewriting of Sec. 3.4.3 fuses them: Gemm with no transposition
+// and unit scale factors.
+extern "C" onnxb_status onnx_matmul_add_run(int64_t M, int64_t N, int64_t K, const float *A, const float *B,
+                                            const float *C, int c_rank, const int64_t *c_dims, int fuse_relu,
+                                            float *Y, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return onnx_gemm_run(0, 0, 1.0f, 1.0f, M, N, K, A, B, C, c_rank, c_dims, fuse_relu, Y, workspace, workspace_bytes,
+                         cuda_stream);
+}

@@ -347,6 +347,24 @@ def test_sweep_index_mapping_on_full_batch(binding):
             assert np.array_equal(got[:, m], want), (C, HW, m)
 
 
+@pytest.mark.parametrize("shape,c_shape", [((64, 1000, 2048), (1000,)), ((130, 70, 300), (130, 1)), ((33, 40, 20), None)])
+def test_matmul_add_entry(binding, shape, c_shape):
+    """MatMul + Add through the fused entry (Sec. 3.4.3) against the oracle's Gemm with unit factors,
+    which the CPU pins tie to MatMul followed by Add."""
+    M, N, K = shape
+    rng = np.random.default_rng(M * 7 + N)
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    B = rng.standard_normal((K, N)).astype(np.float32)
+    C = rng.standard_normal(c_shape).astype(np.float32) if c_shape else None
+    dev = torch.device("cuda:0")
+    y = binding.onnx_matmul_add(torch.from_numpy(A).to(dev), torch.from_numpy(B).to(dev),
+                                torch.from_numpy(C).to(dev) if C is not None else None, fuse_relu=True)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == 0
+    want, S = oracle.gemm(A, B, C, relu=True)
+    assert worst_ratio(y.cpu().numpy(), want, S) <= 1.0
+
+
 def test_tf32_mma_rate_probe(binding):
     """The measurement aid returns a plausible figure: never faster than the tensor pipe's ideal
     n/2 cycles per 128 x n x 8 instruction, and within a factor two of it; bad arguments are refused."""
