@@ -208,6 +208,34 @@ onnxb_status onnx_matmul_add_run(int64_t M, int64_t N, int64_t K, const float *A
                                  const float *C, int c_rank, const int64_t *c_dims, int fuse_relu,
                                  float *Y, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * onnx_maxpool2d_shape / onnx_maxpool2d_run - ONNX MaxPool, 2-D, NCHW, dilation 1, ceil_mode 0
+ * (pooling is among the operators the paper lowers, Sec. 4.1; both of its models use it, Sec. 4.2):
+ *
+ *   Y[n,c,p,q] = max over r < kH, s < kW of X[n,c, p*sh + r - pt, q*sw + s - pl]
+ *
+ * where positions outside the image do not take part (the padding value is minus infinity),
+ * P = floor((H + pt + pb - kH) / sh) + 1 and Q likewise.  x_dims = {N,C,H,W}; kernel_shape = {kH,kW};
+ * pads = {h_begin, w_begin, h_end, w_end} or NULL for none; strides = {sh, sw}, NULL or 0 = 1.
+ * All four arrays are host memory.  X [N,C,H,W] and Y [N,C,P,Q] are caller-owned device memory, dense;
+ * the kernel is enqueued on cuda_stream, nothing is allocated or synchronised.  The result is exact.
+ * Errors: ERR_NULL; ERR_SHAPE (non-positive sizes, negative pads, a pad as large as the kernel,
+ * kernel larger than the padded input); ERR_UNSUPPORTED (more than 2^31-1 elements); ERR_CUDA.
+ * onnx_maxpool2d_shape only computes y_dims (host).
+ */
+onnxb_status onnx_maxpool2d_shape(const int64_t x_dims[4], const int64_t kernel_shape[2], const int64_t pads[4],
+                                  const int64_t strides[2], int64_t y_dims[4]);
+onnxb_status onnx_maxpool2d_run(const int64_t x_dims[4], const int64_t kernel_shape[2], const int64_t pads[4],
+                                const int64_t strides[2], const float *X, float *Y, void *cuda_stream);
+
+/*
+ * onnx_global_average_pool_run - ONNX GlobalAveragePool (ResNet50's last pooling, Sec. 4.2):
+ * Y[n,c,0,0] = mean over h, w of X[n,c,h,w].  x_dims = {N,C,H,W} (host); X device [N,C,H,W],
+ * Y device [N,C,1,1]; fp32 accumulation (32 partial sums per plane, then a tree).  Enqueued on
+ * cuda_stream; allocates and synchronises nothing.  Errors: ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_CUDA.
+ */
+onnxb_status onnx_global_average_pool_run(const int64_t x_dims[4], const float *X, float *Y, void *cuda_stream);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char *onnxb_status_string(onnxb_status status);
 

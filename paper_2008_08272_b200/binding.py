@@ -25,6 +25,7 @@ EXPORTS = [
     "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
     "onnxb_probe_tf32_mma_rate", "onnx_matmul_add_run",
+    "onnx_maxpool2d_shape", "onnx_maxpool2d_run", "onnx_global_average_pool_run",
 ]
 
 
@@ -86,6 +87,13 @@ def load(build_if_missing: bool = True):
     lib.onnx_matmul_add_run.restype = ctypes.c_int
     lib.onnx_matmul_add_run.argtypes = [i64, i64, i64, vp, vp, vp, ctypes.c_int, ctypes.POINTER(i64), ctypes.c_int, vp,
                                         vp, sz, vp]
+    p64 = ctypes.POINTER(i64)
+    lib.onnx_maxpool2d_shape.restype = ctypes.c_int
+    lib.onnx_maxpool2d_shape.argtypes = [p64, p64, p64, p64, p64]
+    lib.onnx_maxpool2d_run.restype = ctypes.c_int
+    lib.onnx_maxpool2d_run.argtypes = [p64, p64, p64, p64, vp, vp, vp]
+    lib.onnx_global_average_pool_run.restype = ctypes.c_int
+    lib.onnx_global_average_pool_run.argtypes = [p64, vp, vp, vp]
     lib.onnxb_status_string.restype = ctypes.c_char_p
     lib.onnxb_status_string.argtypes = [ctypes.c_int]
     lib.onnxb_last_device_status.restype = ctypes.c_int
@@ -292,4 +300,39 @@ def onnx_matmul_add(A, B, C=None, *, fuse_relu=False, Y=None, workspace=None, st
     _check(lib.onnx_matmul_add_run(M, N, K, _dev_ptr(A, "A"), _dev_ptr(B, "B"), _dev_ptr(C, "C", allow_none=True),
                                    c_rank, c_dims, int(bool(fuse_relu)), _dev_ptr(Y, "Y"), ws_ptr, ws_len,
                                    _stream_ptr(stream)), "onnx_matmul_add_run")
+    return Y
+
+
+def _i64(values, n):
+    if values is None:
+        return None
+    return (ctypes.c_int64 * n)(*[int(v) for v in values])
+
+
+def maxpool2d_shape(x_shape, kernel_shape, pads=None, strides=None):
+    """``onnx_maxpool2d_shape``: output dims of ONNX MaxPool (host only)."""
+    y = (ctypes.c_int64 * 4)()
+    _check(load().onnx_maxpool2d_shape(_i64(x_shape, 4), _i64(kernel_shape, 2), _i64(pads, 4), _i64(strides, 2), y),
+           "onnx_maxpool2d_shape")
+    return tuple(int(v) for v in y)
+
+
+def onnx_maxpool2d(X, kernel_shape, *, pads=None, strides=None, Y=None, stream=None):
+    """``onnx_maxpool2d_run``: ONNX MaxPool (2-D, NCHW, dilation 1, ceil_mode 0)."""
+    import torch
+    y_shape = maxpool2d_shape(tuple(X.shape), kernel_shape, pads, strides)
+    if Y is None:
+        Y = torch.empty(y_shape, dtype=torch.float32, device=X.device)
+    _check(load().onnx_maxpool2d_run(_i64(tuple(X.shape), 4), _i64(kernel_shape, 2), _i64(pads, 4), _i64(strides, 2),
+                                     _dev_ptr(X, "X"), _dev_ptr(Y, "Y"), _stream_ptr(stream)), "onnx_maxpool2d_run")
+    return Y
+
+
+def onnx_global_average_pool(X, *, Y=None, stream=None):
+    """``onnx_global_average_pool_run``: Y[n,c,0,0] = mean of X[n,c,:,:]."""
+    import torch
+    if Y is None:
+        Y = torch.empty((X.shape[0], X.shape[1], 1, 1), dtype=torch.float32, device=X.device)
+    _check(load().onnx_global_average_pool_run(_i64(tuple(X.shape), 4), _dev_ptr(X, "X"), _dev_ptr(Y, "Y"),
+                                               _stream_ptr(stream)), "onnx_global_average_pool_run")
     return Y
