@@ -465,6 +465,53 @@ def run_probe_tf32():
     return 0
 
 
+def run_pool():
+    """ResNet-50's MaxPool (3x3, stride 2, pad 1 on [64,64,112,112]) and GlobalAveragePool ([64,2048,7,7]):
+    device time per launch with L2 flushed before each (ten flush+run pairs minus ten flushes), against
+    the measured HBM copy bandwidth.  One JSON line."""
+    import torch
+    from paper_2008_08272_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    binding.load(build_if_missing=False)
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(fn, reps=10):
+        def once(with_run):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                flush.zero_()
+                if with_run:
+                    fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / reps
+        fn()
+        return min(once(True) for _ in range(3)) - min(once(False) for _ in range(3))
+
+    out = {"metric": "pooling operators, device time per launch (L2 flushed)", "unit": "us", "data": "synthetic",
+           "hbm_peak_gbs": peaks["hbm_gbs"], "ops": {}}
+    x = torch.rand((64, 64, 112, 112), device=dev)
+    y = torch.empty((64, 64, 56, 56), device=dev)
+    us = timed(lambda: binding.onnx_maxpool2d(x, (3, 3), pads=(1, 1, 1, 1), strides=(2, 2), Y=y))
+    nbytes = 4 * (x.numel() + y.numel())
+    out["ops"]["maxpool_3x3_s2_64x64x112x112"] = {"us": round(us, 1), "gbs": round(nbytes / us / 1e3, 1),
+                                                  "frac_of_hbm_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 3)}
+    x2 = torch.rand((64, 2048, 7, 7), device=dev)
+    y2 = torch.empty((64, 2048, 1, 1), device=dev)
+    us = timed(lambda: binding.onnx_global_average_pool(x2, Y=y2))
+    nbytes = 4 * (x2.numel() + y2.numel())
+    out["ops"]["global_average_pool_64x2048x7x7"] = {"us": round(us, 1), "gbs": round(nbytes / us / 1e3, 1),
+                                                     "frac_of_hbm_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 3)}
+    print(json.dumps(out))
+    return 0
+
+
 def measured_clock_max_mhz():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -483,6 +530,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: run only the convolutions whose name contains this")
     ap.add_argument("--batch", type=int, default=64, help="images per convolution (the benchmark proper uses 64)")
+    ap.add_argument("--pool", action="store_true",
+                    help="time the two pooling operators at ResNet-50 batch-64 sizes instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
                     help="measure the issue-rate ceiling of the TF32 tensor-core instruction instead of the step")
     args = ap.parse_args()
@@ -491,6 +540,8 @@ def main():
         return run_reference(args)
     if args.probe_tf32:
         return run_probe_tf32()
+    if args.pool:
+        return run_pool()
     return run_ours(args)
 
 
