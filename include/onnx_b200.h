@@ -138,6 +138,19 @@ onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t desc, const float *X, const flo
                              const float *B, float *Y, void *workspace, size_t workspace_bytes,
                              void *cuda_stream);
 
+/*
+ * onnx_conv2d_add_run - Conv, then Add of a second tensor, then the descriptor's Relu, in one
+ * pass: Y = relu?( Conv(X, W) + B + R ).  This is a residual connection written the way the
+ * compiler's fusion of a single-use producer into its consumer leaves it (Sec. 3.4.3; elementwise
+ * Add is the paper's running example, Sec. 3.2): the convolution's output is never written and
+ * read back.  R: device, same shape and layout as Y ([N, M, P, Q], dense, 16-byte aligned), read
+ * only, must not overlap Y; every other argument and error exactly as for onnx_conv2d_run
+ * (ERR_NULL when R is NULL).  The addition is one fp32 add per element before the Relu.
+ */
+onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t desc, const float *X, const float *W, const float *B,
+                                 const float *R, float *Y, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream);
+
 void onnx_conv2d_desc_destroy(onnxb_conv2d_desc_t desc);
 
 /*

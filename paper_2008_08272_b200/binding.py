@@ -25,7 +25,7 @@ EXPORTS = [
     "onnx_gemm_workspace_bytes", "onnx_gemm_run", "onnxb_status_string",
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
     "onnxb_probe_tf32_mma_rate", "onnx_matmul_add_run",
-    "onnx_maxpool2d_shape", "onnx_maxpool2d_run", "onnx_global_average_pool_run",
+    "onnx_maxpool2d_shape", "onnx_maxpool2d_run", "onnx_global_average_pool_run", "onnx_conv2d_add_run",
 ]
 
 
@@ -73,6 +73,8 @@ def load(build_if_missing: bool = True):
     lib.onnx_conv2d_desc_query_kernel.argtypes = [vp]
     lib.onnx_conv2d_run.restype = ctypes.c_int
     lib.onnx_conv2d_run.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.onnx_conv2d_add_run.restype = ctypes.c_int
+    lib.onnx_conv2d_add_run.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.onnx_conv2d_run_static.restype = ctypes.c_int
     lib.onnx_conv2d_run_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.onnx_conv2d_static_scratch_bytes.restype = sz
@@ -181,6 +183,20 @@ class Conv2dDesc:
         _check(self._lib.onnx_conv2d_run(self._h, _dev_ptr(X, "X"), _dev_ptr(W, "W"),
                                          _dev_ptr(B, "B", allow_none=True), _dev_ptr(Y, "Y"),
                                          ws_ptr, ws_len, _stream_ptr(stream)), "onnx_conv2d_run")
+        return Y
+
+    def run_add(self, X, W, B, R, Y=None, workspace=None, stream=None):
+        """``onnx_conv2d_add_run``: Y = relu?(Conv(X, W) + B + R), R shaped like Y (a residual connection)."""
+        import torch
+        if Y is None:
+            Y = torch.empty(self.y_shape, dtype=torch.float32, device=X.device)
+        if workspace is None and self.workspace_bytes:
+            workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=X.device)
+        ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+        ws_len = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        _check(self._lib.onnx_conv2d_add_run(self._h, _dev_ptr(X, "X"), _dev_ptr(W, "W"),
+                                             _dev_ptr(B, "B", allow_none=True), _dev_ptr(R, "R"), _dev_ptr(Y, "Y"),
+                                             ws_ptr, ws_len, _stream_ptr(stream)), "onnx_conv2d_add_run")
         return Y
 
     def run_static(self, X, W, B=None, Y=None, stream=None):

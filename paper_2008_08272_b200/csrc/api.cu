@@ -24,7 +24,8 @@ unsigned int *device_status_ptr() {
 
 // A 1x1, stride-1, unpadded, ungrouped convolution is one GEMM per image:
 // Y[n] (M x HW) = W (M x C) * X[n] (C x HW), with W K-major and X[n] pixel-major.
-static TcGemmProblem conv1x1_as_gemm(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y) {
+static TcGemmProblem conv1x1_as_gemm(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+                                     const float *R = nullptr) {
     TcGemmProblem t{};
     const long long HW = (long long)g.H * g.W;
     t.M = g.M; t.N = (int)HW; t.K = g.C; t.batch = g.N;
@@ -33,7 +34,7 @@ static TcGemmProblem conv1x1_as_gemm(const ConvGeom &g, const float *X, const fl
     t.a_ld = g.C; t.b_ld = HW; t.a_bs = 0; t.b_bs = (long long)g.C * HW;
     t.a_batched = 0; t.b_batched = 1;
     t.alpha = 1.f; t.beta = 0.f; t.C = nullptr;
-    t.row_bias = B; t.relu = g.relu;
+    t.row_bias = B; t.relu = g.relu; t.residual = R;
     t.Y = Y; t.y_ld = HW; t.y_bs = (long long)g.M * HW;
     return t;
 }
@@ -64,7 +65,7 @@ static long long gather_pitch(const ConvGeom &g) {
 }
 
 static TcGemmProblem conv1x1_gathered_as_gemm(const ConvGeom &g, const float *Xg, const float *W, const float *B,
-                                              float *Y) {
+                                              float *Y, const float *R = nullptr) {
     TcGemmProblem t{};
     const long long PQ = (long long)g.P * g.Q, pitch = gather_pitch(g);
     const bool merged = gather_merged(g);
@@ -73,7 +74,7 @@ static TcGemmProblem conv1x1_gathered_as_gemm(const ConvGeom &g, const float *Xg
     t.a_mn_major = 0; t.b_mn_major = 1;
     t.a_ld = g.C; t.b_ld = pitch; t.a_bs = 0; t.a_batched = 0;
     t.alpha = 1.f; t.beta = 0.f; t.C = nullptr;
-    t.row_bias = B; t.relu = g.relu;
+    t.row_bias = B; t.relu = g.relu; t.residual = R;
     t.Y = Y; t.y_ld = PQ;
     if (merged) {
         t.N = (int)(PQ * g.N); t.batch = 1; t.b_bs = 0; t.b_batched = 0; t.y_bs = 0;
@@ -102,10 +103,11 @@ size_t conv_gather_workspace_bytes(const ConvGeom &g) {
 
 static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
-extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, const float *W,
-                                        const float *B, float *Y, void *workspace, size_t workspace_bytes,
-                                        void *cuda_stream) {
+static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const float *W, const float *B,
+                                    const float *R, float *Y, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream) {
     if (!d || !X || !W || !Y) return ONNXB_ERR_NULL;
+    if (misaligned(R)) return ONNXB_ERR_UNSUPPORTED;
     if ((d->g.has_bias != 0) != (B != nullptr)) return ONNXB_ERR_NULL;
     if (d->workspace_bytes > 0 && (!workspace || workspace_bytes < d->workspace_bytes)) return ONNXB_ERR_WORKSPACE;
     if (misaligned(X) || misaligned(W) || misaligned(B) || misaligned(Y) || misaligned(workspace))
@@ -114,28 +116,43 @@ extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, c
     int err;
     switch (d->family) {
         case ONNXB_KERNEL_SIMT_DEPTHWISE:
-            err = launch_simt_depthwise(d->g, X, W, B, Y, cuda_stream);
+            err = launch_simt_depthwise(d->g, X, W, B, R, Y, cuda_stream);
             break;
         case ONNXB_KERNEL_SIMT_DIRECT:
-            err = launch_simt_conv(d->g, X, W, B, Y, cuda_stream);
+            err = launch_simt_conv(d->g, X, W, B, R, Y, cuda_stream);
             break;
         case ONNXB_KERNEL_MMA_GEMM:
-            err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y), cuda_stream);
+            err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y, R), cuda_stream);
             break;
         case ONNXB_KERNEL_MMA_GATHER_GEMM:
             err = launch_gather1x1(d->g, X, static_cast<float *>(workspace), gather_pitch(d->g), gather_merged(d->g),
                                    cuda_stream);
             if (err == 0)
-                err = launch_tc_gemm(conv1x1_gathered_as_gemm(d->g, static_cast<const float *>(workspace), W, B, Y),
+                err = launch_tc_gemm(conv1x1_gathered_as_gemm(d->g, static_cast<const float *>(workspace), W, B, Y, R),
                                      cuda_stream);
             break;
         case ONNXB_KERNEL_MMA_IMPLICIT:
-            err = launch_tc_conv(d->plan, X, W, B, Y, workspace, cuda_stream);
+            err = launch_tc_conv(d->plan, X, W, B, R, Y, workspace, cuda_stream);
             break;
         default:
             return ONNXB_ERR_UNSUPPORTED;
     }
     return err == 0 ? ONNXB_OK : ONNXB_ERR_CUDA;
+}
+
+extern "C" onnxb_status onnx_conv2d_run(onnxb_conv2d_desc_t d, const float *X, const float *W,
+                                        const float *B, float *Y, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream) {
+    return conv2d_run_impl(d, X, W, B, nullptr, Y, workspace, workspace_bytes, cuda_stream);
+}
+
+// Conv followed by Add (a residual connection) and the descriptor's Relu, in one pass: the single-use
+// producer/consumer fusion of Sec. 3.4.3 applied to Conv -> Add -> Relu.
+extern "C" onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t d, const float *X, const float *W, const float *B,
+                                            const float *R, float *Y, void *workspace, size_t workspace_bytes,
+                                            void *cuda_stream) {
+    if (!R) return ONNXB_ERR_NULL;
+    return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" size_t onnx_gemm_workspace_bytes(int, int, int64_t, int64_t, int64_t) { return 0; }

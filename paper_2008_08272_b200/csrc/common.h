@@ -39,9 +39,10 @@ inline void count_launch(int n = 1) { g_launches.fetch_add((uint64_t)n, std::mem
 int kernel_override();   // -1 = automatic
 
 // SIMT family (simt_conv.cu / simt_gemm.cu).  All return a cudaError_t as int.
-int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+// R (everywhere below): optional addend with Y's shape, added before Relu (a residual connection); may be NULL.
+int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
                      void *stream);
-int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
                           void *stream);
 bool simt_depthwise_supports(const ConvGeom &g);
 bool conv_fits_mma_gemm(const ConvGeom &g);
@@ -51,7 +52,7 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
 // implicit-GEMM tensor-core convolution (tc_conv.cu)
 bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan, bool forced = false);
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan);
-int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, float *Y,
+int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, const float *R, float *Y,
                    void *workspace, void *stream);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
 
 struct GemmProblem {

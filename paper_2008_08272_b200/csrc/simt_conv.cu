@@ -23,7 +23,8 @@ constexpr int kDirectChunk = 256;     // reduction terms staged in shared memory
 template <int MT>
 __global__ void __launch_bounds__(kDirectThreads)
 conv2d_direct_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
-                     const float *__restrict__ B, float *__restrict__ Y, int pixel_tiles, int m_tiles_per_group) {
+                     const float *__restrict__ B, const float *__restrict__ R, float *__restrict__ Y, int pixel_tiles,
+                     int m_tiles_per_group) {
     __shared__ float wsm[MT * kDirectChunk];
 
     const int tile = blockIdx.x % pixel_tiles;
@@ -85,8 +86,10 @@ conv2d_direct_kernel(const ConvGeom g, const float *__restrict__ X, const float 
                 const int m = m0 + j;
                 if (m < m_end) {
                     float v = acc[j] + (B ? __ldg(B + m) : 0.f);
+                    const size_t yi = ((size_t)n * g.M + m) * PQ + pix;
+                    if (R) v += __ldg(R + yi);              // residual addend at Y's own position
                     if (g.relu) v = v > 0.f ? v : 0.f;
-                    Y[((size_t)n * g.M + m) * PQ + pix] = v;
+                    Y[yi] = v;
                 }
             }
         }
@@ -103,7 +106,8 @@ constexpr int kDwTP = 32, kDwTQ = 32, kDwRows = 4, kDwThreads = kDwTQ * (kDwTP /
 
 __global__ void __launch_bounds__(kDwThreads)
 conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
-                        const float *__restrict__ B, float *__restrict__ Y, int q_tiles, int p_tiles,
+                        const float *__restrict__ B, const float *__restrict__ R, float *__restrict__ Y, int q_tiles,
+                        int p_tiles,
                         int in_rows, int in_cols, int pitch) {
     extern __shared__ float tile[];           // [in_rows][pitch] then weights [kH*kW]
     float *wsm = tile + in_rows * pitch;
@@ -152,8 +156,10 @@ conv2d_depthwise_kernel(const ConvGeom g, const float *__restrict__ X, const flo
         const int p = p0 + tp + k;
         if (p < g.P) {
             float v = acc[k] + bias;
+            const size_t yi = ((size_t)plane * g.P + p) * g.Q + q;
+            if (R) v += __ldg(R + yi);
             if (g.relu) v = v > 0.f ? v : 0.f;
-            Y[((size_t)plane * g.P + p) * g.Q + q] = v;
+            Y[yi] = v;
         }
     }
 }
@@ -225,8 +231,8 @@ gather1x1_vec_kernel(const float4 *__restrict__ X4, float4 *__restrict__ Xg4, un
 template <int KH, int KW, bool VEC>
 __global__ void __launch_bounds__(256)
 conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
-                             const float *__restrict__ B, float *__restrict__ Y, unsigned items, unsigned Q4,
-                             unsigned P2, double inv_Q4, double inv_P2) {
+                             const float *__restrict__ B, const float *__restrict__ R, float *__restrict__ Y,
+                             unsigned items, unsigned Q4, unsigned P2, double inv_Q4, double inv_P2) {
     constexpr int WIN = KW + 3;                // input columns a strip of 4 outputs touches
     const unsigned i = blockIdx.x * 256u + threadIdx.x;
     if (i >= items) return;
@@ -290,6 +296,11 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
     for (int k = 0; k < 2; ++k) {
         float *a = k ? acc1 : acc0;
         if (p0 + k >= g.P) break;
+        if (R) {
+            const float *rr = R + (yp - Y) + (size_t)k * g.Q;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if (q0 + j < g.Q) a[j] += __ldg(rr + j);
+        }
         if (g.relu) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) a[j] = a[j] > 0.f ? a[j] : 0.f;
@@ -305,7 +316,8 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
 }
 
 template <int KH, int KW>
-int launch_depthwise_unit(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y, cudaStream_t st) {
+int launch_depthwise_unit(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
+                          cudaStream_t st) {
     const unsigned Q4 = (unsigned)((g.Q + 3) / 4), P2 = (unsigned)((g.P + 1) / 2);
     const long long items = (long long)g.N * g.C * P2 * Q4;
     const unsigned blocks = (unsigned)((items + 255) / 256);
@@ -313,10 +325,10 @@ int launch_depthwise_unit(const ConvGeom &g, const float *X, const float *W, con
     const bool vec = g.pl == 1 && g.W % 4 == 0 && g.Q % 4 == 0 &&
                      (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15) == 0;
     if (vec)
-        conv2d_depthwise_unit_kernel<KH, KW, true><<<blocks, 256, 0, st>>>(g, X, W, B, Y, (unsigned)items, Q4, P2,
+        conv2d_depthwise_unit_kernel<KH, KW, true><<<blocks, 256, 0, st>>>(g, X, W, B, R, Y, (unsigned)items, Q4, P2,
                                                                             1.0 / (double)Q4, 1.0 / (double)P2);
     else
-        conv2d_depthwise_unit_kernel<KH, KW, false><<<blocks, 256, 0, st>>>(g, X, W, B, Y, (unsigned)items, Q4, P2,
+        conv2d_depthwise_unit_kernel<KH, KW, false><<<blocks, 256, 0, st>>>(g, X, W, B, R, Y, (unsigned)items, Q4, P2,
                                                                              1.0 / (double)Q4, 1.0 / (double)P2);
     count_launch();
     return (int)cudaGetLastError();
@@ -374,11 +386,11 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
     return (int)cudaGetLastError();
 }
 
-int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
                           void *stream) {
     if (depthwise_unit_fits(g)) {
-        if (g.kH == 3) return launch_depthwise_unit<3, 3>(g, X, W, B, Y, (cudaStream_t)stream);
-        return launch_depthwise_unit<5, 5>(g, X, W, B, Y, (cudaStream_t)stream);
+        if (g.kH == 3) return launch_depthwise_unit<3, 3>(g, X, W, B, R, Y, (cudaStream_t)stream);
+        return launch_depthwise_unit<5, 5>(g, X, W, B, R, Y, (cudaStream_t)stream);
     }
     int rows, cols, pitch;
     depthwise_window(g, rows, cols, pitch);
@@ -390,13 +402,13 @@ int launch_simt_depthwise(const ConvGeom &g, const float *X, const float *W, con
         if (e != cudaSuccess) return (int)e;
     }
     const unsigned blocks = (unsigned)((long long)q_tiles * p_tiles * g.N * g.C);
-    conv2d_depthwise_kernel<<<blocks, kDwThreads, smem, (cudaStream_t)stream>>>(g, X, W, B, Y, q_tiles, p_tiles, rows,
+    conv2d_depthwise_kernel<<<blocks, kDwThreads, smem, (cudaStream_t)stream>>>(g, X, W, B, R, Y, q_tiles, p_tiles, rows,
                                                                               cols, pitch);
     count_launch();
     return (int)cudaGetLastError();
 }
 
-int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const float *B, float *Y,
+int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
                      void *stream) {
     const long long PQ = (long long)g.P * g.Q;
     const int pixel_tiles = (int)((PQ + kDirectThreads - 1) / kDirectThreads);
@@ -408,11 +420,11 @@ int launch_simt_conv(const ConvGeom &g, const float *X, const float *W, const fl
     dim3 grid((unsigned)gx, (unsigned)(m_tiles > 65535 ? 65535 : m_tiles), 1);
     cudaStream_t st = (cudaStream_t)stream;
     if (MT == 8)
-        conv2d_direct_kernel<8><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+        conv2d_direct_kernel<8><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, R, Y, pixel_tiles, m_tiles_per_group);
     else if (MT == 4)
-        conv2d_direct_kernel<4><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+        conv2d_direct_kernel<4><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, R, Y, pixel_tiles, m_tiles_per_group);
     else
-        conv2d_direct_kernel<1><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, Y, pixel_tiles, m_tiles_per_group);
+        conv2d_direct_kernel<1><<<grid, kDirectThreads, 0, st>>>(g, X, W, B, R, Y, pixel_tiles, m_tiles_per_group);
     count_launch();
     return (int)cudaGetLastError();
 }

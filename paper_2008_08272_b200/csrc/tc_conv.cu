@@ -136,11 +136,13 @@ __global__ void pack_weights_kernel(const TcConvPlan g, const float *__restrict_
 __device__ __forceinline__ int cb_rotation(long long tile, int ncb) { return (int)((tile * 5 + 3) % ncb); }
 
 // ------------------------------------------------------------------ main kernel
-template <int kCtas>
+// kAdd: the epilogue also adds a tensor laid out like Y (a residual connection) before the Relu.  A
+// separate instantiation, so that the plain kernel's register allocation is not disturbed.
+template <int kCtas, bool kAdd>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, const float *__restrict__ X,
-               const float *__restrict__ Wpk, const float *__restrict__ bias, float *__restrict__ Y,
-               unsigned int *err) {
+               const float *__restrict__ Wpk, const float *__restrict__ bias, const float *__restrict__ R,
+               float *__restrict__ Y, unsigned int *err) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler
     // keeps treating everything derived from it as shared memory (LDS/STS, not generic accesses)
@@ -553,8 +555,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float x = __uint_as_float(v[j]) + __shfl_sync(0xffffffffu, bl, j);
+                    const bool live = valid && mg0 + j < m_lim;
+                    if (kAdd && live) x += __ldg(R + (yp - Y));             // residual addend at Y's own position
                     if (g.relu) x = fmaxf(x, 0.f);
-                    if (valid && mg0 + j < m_lim) *yp = x;
+                    if (live) *yp = x;
                     yp += PQ;
                 }
             }
@@ -919,7 +923,7 @@ static int max_pairs(size_t smem) {
     cfg.numAttrs = 1;
     int n = 0;
     (void)smem;
-    if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2>, &cfg) != cudaSuccess || n < 1) {
+    if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2, false>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = tc_host::num_sms() / 2;
     }
@@ -929,7 +933,7 @@ static int max_pairs(size_t smem) {
 
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan) { return (size_t)plan.packed_floats * 4; }
 
-int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, float *Y,
+int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, const float *R, float *Y,
                    void *workspace, void *stream) {
     using namespace tc_host;
     cudaStream_t st = (cudaStream_t)stream;
@@ -958,8 +962,10 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     const size_t smem = 1024 + (size_t)plan.na_stages * plan.a_stage_bytes + (size_t)plan.nr_stages * plan.raw_stage_bytes +
                         (size_t)plan.nb_stages * plan.b_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
     const bool pair = plan.ctas == 2;
-    cudaError_t e = cudaFuncSetAttribute(pair ? tc_conv_kernel<2> : tc_conv_kernel<1>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    const bool add = R != nullptr;
+    auto kern = pair ? (add ? tc_conv_kernel<2, true> : tc_conv_kernel<2, false>)
+                     : (add ? tc_conv_kernel<1, true> : tc_conv_kernel<1, false>);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return (int)e;
     const int sms = num_sms();
     // persistent: one CTA per SM; pairs are clusters of two neighbouring SMs
@@ -973,10 +979,10 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
             plan.raw_stage_bytes, plan.b_stage_bytes, plan.nb_stages, smem);
 #endif
     const cudaError_t le =
-        pair ? launch_pdl_cluster(tc_conv_kernel<2>, 2, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
-                                  reinterpret_cast<const float *>(workspace), B, Y, err)
-             : launch_pdl(tc_conv_kernel<1>, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
-                          reinterpret_cast<const float *>(workspace), B, Y, err);
+        pair ? launch_pdl_cluster(kern, 2, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+                                  reinterpret_cast<const float *>(workspace), B, R, Y, err)
+             : launch_pdl(kern, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+                          reinterpret_cast<const float *>(workspace), B, R, Y, err);
     count_launch();
     return (int)le;
 }

@@ -69,6 +69,7 @@ struct Params {
     const float *C;            // optional addend, element strides below (0 = broadcast)
     long long c_si, c_sj, c_sb;
     const float *row_bias;     // optional per-row addend (convolution bias)
+    const float *R;            // optional addend laid out exactly like Y (a residual connection), added before Relu
     int relu;
     // MN-major B in one copy per stage: a 4-D view (32 columns of a block, K row, block of 32 columns,
     // batch) lets a single box carry all of a tile's 32-column blocks in the order the MMA wants them.
@@ -296,10 +297,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 auto finish = [&](const uint32_t (&v)[32], int chunk) {
                     const int col0 = tn * p.BN + chunk * 32;
                     float f[32];
-                    if (p.C == nullptr) {
+                    if (p.C == nullptr && p.R == nullptr) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
+                            f[j] = p.relu ? fmaxf(x, 0.f) : x;
+                        }
+                    } else if (p.C == nullptr) {
+                        // residual addend: the element of R at Y's own position (this lane's row, 32
+                        // consecutive columns; with split columns the position is worked out per element)
+                        const bool row_ok = row < p.M;
+                        const float *rp = p.R + b * p.y_sb + (long long)row * p.y_ld;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
+                            const int col = col0 + j;
+                            if (row_ok && col < p.N) {
+                                long long coff = col;
+                                if (p.y_split > 0) {
+                                    const int grp = col / p.y_split;
+                                    coff = (long long)grp * p.y_group + (col - grp * p.y_split);
+                                }
+                                x += __ldg(rp + coff);
+                            }
                             f[j] = p.relu ? fmaxf(x, 0.f) : x;
                         }
                     } else {
@@ -548,6 +568,7 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
     p.row_bias = g.row_bias; p.relu = g.relu;
+    p.R = g.C ? nullptr : g.residual;
     p.Y = g.Y; p.y_ld = g.y_ld; p.y_sb = g.y_bs;
     p.y_split = g.y_split; p.y_group = g.y_group_stride;
     p.y_tma = g.y_split == 0 && (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);

@@ -21,6 +21,7 @@ struct TcGemmProblem {
     const float *C;
     long long c_si, c_sj, c_sb;
     const float *row_bias;
+    const float *residual;   // optional addend with Y's own layout, added before Relu (ignored when C is given)
     int relu;
     float *Y;
     long long y_ld, y_bs;

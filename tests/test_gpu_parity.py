@@ -365,6 +365,49 @@ def test_matmul_add_entry(binding, shape, c_shape):
     assert worst_ratio(y.cpu().numpy(), want, S) <= 1.0
 
 
+# Conv + Add + Relu in one pass, one case per kernel family (and both GEMM store paths)
+ADD_CASES = [
+    dict(x=(2, 64, 28, 28), w=(256, 64, 1, 1)),                                   # GEMM, TMA stores, CTA pairs
+    dict(x=(3, 96, 14, 14), w=(72, 96, 1, 1)),                                    # GEMM, one CTA per tile
+    dict(x=(5, 128, 7, 7), w=(320, 128, 1, 1)),                                   # gathered, merged columns
+    dict(x=(2, 64, 28, 28), w=(128, 64, 1, 1), strides=(2, 2)),                   # gathered, per image
+    dict(x=(2, 32, 30, 30), w=(48, 32, 3, 3), pads=(1, 1, 1, 1)),                 # implicit GEMM
+    dict(x=(9, 32, 7, 7), w=(144, 32, 3, 3), pads=(1, 1, 1, 1)),                  # implicit GEMM, pair tiles
+    dict(x=(2, 4, 13, 11), w=(6, 4, 3, 3), pads=(1, 1, 1, 1)),                    # SIMT direct
+    dict(x=(2, 24, 28, 28), w=(24, 1, 3, 3), pads=(1, 1, 1, 1), group=24),        # depthwise, unit stride
+    dict(x=(2, 24, 27, 29), w=(24, 1, 5, 5), pads=(2, 2, 2, 2), strides=(2, 2), group=24),   # depthwise, general
+]
+
+
+@pytest.mark.parametrize("c", ADD_CASES, ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+@pytest.mark.parametrize("relu", [False, True])
+def test_conv_add_relu_fused(binding, c, relu):
+    """Y = relu?(Conv(X, W) + B + R) against the oracle's convolution plus the addend, Relu applied last."""
+    rng = np.random.default_rng(515)
+    X = rng.standard_normal(c["x"]).astype(np.float32)
+    fan = c["w"][1] * c["w"][2] * c["w"][3]
+    W = (rng.standard_normal(c["w"]) * np.sqrt(2.0 / fan)).astype(np.float32)
+    B = (rng.standard_normal((c["w"][0],)) * 0.1).astype(np.float32)
+    kw = dict(pads=c.get("pads", (0, 0, 0, 0)), strides=c.get("strides", (1, 1)), group=c.get("group", 1))
+    conv, S = oracle.conv2d(X, W, B, relu=False, **kw)
+    R = rng.standard_normal(conv.shape).astype(np.float32)
+    want = conv + R.astype(np.float64)
+    if relu:
+        want = np.maximum(want, 0.0)
+    dev = torch.device("cuda:0")
+    d = binding.Conv2dDesc(tuple(X.shape), tuple(W.shape), has_bias=True, fuse_relu=relu, **kw)
+    numel = want.size
+    buf = torch.full((numel + 128,), 4321.0, dtype=torch.float32, device=dev)
+    Y = buf[64:64 + numel].view(want.shape)
+    d.run_add(torch.from_numpy(X).to(dev), torch.from_numpy(W).to(dev), torch.from_numpy(B).to(dev),
+              torch.from_numpy(R).to(dev), Y=Y)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == 0
+    assert bool((buf[:64] == 4321.0).all()) and bool((buf[64 + numel:] == 4321.0).all()), "store outside Y"
+    d.close()
+    assert worst_ratio(Y.cpu().numpy(), want, S) <= 1.0
+
+
 def test_tf32_mma_rate_probe(binding):
     """The measurement aid returns a plausible figure: never faster than the tensor pipe's ideal
     n/2 cycles per 128 x n x 8 instruction, and within a factor two of it; bad arguments are refused."""
