@@ -465,6 +465,43 @@ def run_probe_tf32():
     return 0
 
 
+def run_model(args):
+    """Chained ResNet-50 v1 inference at --batch images (synthetic weights): 53 convolutions with fused
+    bias/Relu and fused residual Add, the two pools and the classifier Gemm, enqueued back to back on one
+    stream.  Device time per forward pass over --steps passes after --warmup; one JSON line.  This is the
+    figure comparable in kind (not in hardware) with the inference times of the paper's Table 1."""
+    import torch
+    from paper_2008_08272_b200 import binding
+    from paper_2008_08272_b200.resnet50_chain import Resnet50Chain
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    binding.load(build_if_missing=False)
+    net = Resnet50Chain(args.batch, dev)
+    x = torch.rand((args.batch, 3, 224, 224), device=dev)
+    for _ in range(max(args.warmup, 3)):
+        net.forward(x)
+    torch.cuda.synchronize()
+    l0 = binding.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        net.forward(x)
+    e1.record()
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == 0
+    ms = e0.elapsed_time(e1) / args.steps
+    out = {"metric": "ResNet-50 v1 chained inference, device time per forward pass", "value": ms, "unit": "ms",
+           "higher_is_better": False, "batch": args.batch, "images_per_s": round(args.batch / ms * 1e3, 1),
+           "tflops": round(net.flops / (ms * 1e-3) / 1e12, 1), "steps": args.steps, "data": "synthetic",
+           "gpu_launches_per_pass": int((binding.launch_count() - l0) // args.steps),
+           "paper_table1_context": "7.540 s for one image on a 2.3 GHz POWER9 CPU, unoptimised scalar loops"}
+    net.close()
+    print(json.dumps(out))
+    return 0
+
+
 def run_pool():
     """ResNet-50's MaxPool (3x3, stride 2, pad 1 on [64,64,112,112]) and GlobalAveragePool ([64,2048,7,7]):
     device time per launch with L2 flushed before each (ten flush+run pairs minus ten flushes), against
@@ -530,6 +567,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only", default="", help="profiling aid: run only the convolutions whose name contains this")
     ap.add_argument("--batch", type=int, default=64, help="images per convolution (the benchmark proper uses 64)")
+    ap.add_argument("--model", action="store_true",
+                    help="time a chained ResNet-50 v1 forward pass (all operators, one stream) instead of the step")
     ap.add_argument("--pool", action="store_true",
                     help="time the two pooling operators at ResNet-50 batch-64 sizes instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
@@ -542,6 +581,8 @@ def main():
         return run_probe_tf32()
     if args.pool:
         return run_pool()
+    if args.model:
+        return run_model(args)
     return run_ours(args)
 
 

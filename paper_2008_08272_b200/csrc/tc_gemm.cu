@@ -304,24 +304,44 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             f[j] = p.relu ? fmaxf(x, 0.f) : x;
                         }
                     } else if (p.C == nullptr) {
-                        // residual addend: the element of R at Y's own position (this lane's row, 32
-                        // consecutive columns; with split columns the position is worked out per element)
-                        const bool row_ok = row < p.M;
-                        const float *rp = p.R + b * p.y_sb + (long long)row * p.y_ld;
+                        // Residual addend R, laid out like Y.  A lane owns a ROW of the block, but rows are
+                        // far apart in memory, so the block is fetched the other way round: lane = column,
+                        // one coalesced 128-byte read per row, parked in the warp's staging buffer (same
+                        // swizzle as the Y block that follows it there) and read back a row per lane.
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
-                            const int col = col0 + j;
-                            if (row_ok && col < p.N) {
-                                long long coff = col;
-                                if (p.y_split > 0) {
-                                    const int grp = col / p.y_split;
-                                    coff = (long long)grp * p.y_group + (col - grp * p.y_split);
-                                }
-                                x += __ldg(rp + coff);
+                        for (int j = 0; j < 32; ++j) f[j] = fmaf(p.alpha, __uint_as_float(v[j]), rb);
+                        if (p.y_tma && lane == 0) tma_store_wait_read<0>();      // the buffer's last Y block has gone
+                        __syncwarp();
+                        {
+                            const int col = col0 + lane;
+                            long long coff = col;
+                            if (p.y_split > 0) {
+                                const int grp = col / p.y_split;
+                                coff = (long long)grp * p.y_group + (col - grp * p.y_split);
                             }
-                            f[j] = p.relu ? fmaxf(x, 0.f) : x;
+                            const float *rp = p.R + b * p.y_sb + (long long)row0 * p.y_ld + coff;
+                            const int rows = min(32, p.M - row0);
+                            float t[32];
+#pragma unroll
+                            for (int r = 0; r < 32; ++r) {
+                                t[r] = (r < rows && col < p.N) ? __ldg(rp) : 0.f;
+                                rp += p.y_ld;
+                            }
+#pragma unroll
+                            for (int r = 0; r < 32; ++r)
+                                *reinterpret_cast<float *>(buf + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2))) = t[r];
                         }
+                        __syncwarp();
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const float4 t4 = *reinterpret_cast<const float4 *>(buf + lane * 128 + ((c ^ (lane & 7)) << 4));
+                            f[4 * c] += t4.x; f[4 * c + 1] += t4.y; f[4 * c + 2] += t4.z; f[4 * c + 3] += t4.w;
+                        }
+                        if (p.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.f);
+                        }
+                        __syncwarp();                                             // every lane has read its row back
                     } else {
                         // C broadcast: walk one pointer along the row instead of forming 64-bit
                         // products per element (this branch must stay out of the C-less path)
