@@ -484,10 +484,27 @@ def run_model(args):
         net.forward(x)
     torch.cuda.synchronize()
     l0 = binding.launch_count()
+    net.forward(x)
+    per_pass = int(binding.launch_count() - l0)
+    run = lambda: net.forward(x)
+    if args.graph:
+        # the whole pass captured once into a CUDA graph and replayed: the 56 library calls per pass (argument
+        # checks, tensor-map encoding, launches) then cost the host nothing, which is what bounds batch 1
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                net.forward(x)
+        torch.cuda.current_stream().wait_stream(side)
+        run = graph.replay
+        for _ in range(3):
+            run()
+    torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        net.forward(x)
+        run()
     e1.record()
     torch.cuda.synchronize()
     assert binding.last_device_status() == 0
@@ -495,7 +512,7 @@ def run_model(args):
     out = {"metric": "ResNet-50 v1 chained inference, device time per forward pass", "value": ms, "unit": "ms",
            "higher_is_better": False, "batch": args.batch, "images_per_s": round(args.batch / ms * 1e3, 1),
            "tflops": round(net.flops / (ms * 1e-3) / 1e12, 1), "steps": args.steps, "data": "synthetic",
-           "gpu_launches_per_pass": int((binding.launch_count() - l0) // args.steps),
+           "gpu_launches_per_pass": per_pass, "cuda_graph": bool(args.graph),
            "paper_table1_context": "7.540 s for one image on a 2.3 GHz POWER9 CPU, unoptimised scalar loops"}
     net.close()
     print(json.dumps(out))
@@ -569,6 +586,7 @@ def main():
     ap.add_argument("--batch", type=int, default=64, help="images per convolution (the benchmark proper uses 64)")
     ap.add_argument("--model", action="store_true",
                     help="time a chained ResNet-50 v1 forward pass (all operators, one stream) instead of the step")
+    ap.add_argument("--graph", action="store_true", help="with --model: replay the pass from a captured CUDA graph")
     ap.add_argument("--pool", action="store_true",
                     help="time the two pooling operators at ResNet-50 batch-64 sizes instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
