@@ -151,6 +151,27 @@ onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t desc, const float *X, const
                                  const float *R, float *Y, void *workspace, size_t workspace_bytes,
                                  void *cuda_stream);
 
+/*
+ * onnx_conv2d_prepack / onnx_conv2d_run_prepacked - for weights that are constants of the graph
+ * (the usual case in inference; the compiler propagates constants ahead of time, Sec. 3.4.4):
+ * the weight re-layout that onnx_conv2d_run performs at every call is done once.
+ *
+ * onnx_conv2d_prepack writes the packed, TF32-rounded copy of W into `packed` (device, caller-
+ * owned, at least the workspace_bytes of onnx_conv2d_desc_query, 16-byte aligned).  Descriptors
+ * whose kernel reads W directly need no copy: the call then does nothing and returns OK.
+ * onnx_conv2d_run_prepacked computes what onnx_conv2d_run (R == NULL) or onnx_conv2d_add_run
+ * (R != NULL) computes, from that copy.  W must still be passed (the kernels that use no packed
+ * copy read it) and must be the tensor that was packed; `packed` is read only.  workspace /
+ * workspace_bytes: as for onnx_conv2d_run for descriptors that use no packed copy, ignored
+ * (may be NULL / 0) otherwise.  Errors: as the calls they stand for; ERR_WORKSPACE when `packed`
+ * is too small, ERR_NULL when it is missing where needed.
+ */
+onnxb_status onnx_conv2d_prepack(onnxb_conv2d_desc_t desc, const float *W, void *packed, size_t packed_bytes,
+                                 void *cuda_stream);
+onnxb_status onnx_conv2d_run_prepacked(onnxb_conv2d_desc_t desc, const float *X, const float *W, const void *packed,
+                                       const float *B, const float *R, float *Y, void *workspace,
+                                       size_t workspace_bytes, void *cuda_stream);
+
 void onnx_conv2d_desc_destroy(onnxb_conv2d_desc_t desc);
 
 /*

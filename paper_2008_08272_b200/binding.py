@@ -26,6 +26,7 @@ EXPORTS = [
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
     "onnxb_probe_tf32_mma_rate", "onnx_matmul_add_run",
     "onnx_maxpool2d_shape", "onnx_maxpool2d_run", "onnx_global_average_pool_run", "onnx_conv2d_add_run",
+    "onnx_conv2d_prepack", "onnx_conv2d_run_prepacked",
 ]
 
 
@@ -75,6 +76,10 @@ def load(build_if_missing: bool = True):
     lib.onnx_conv2d_run.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
     lib.onnx_conv2d_add_run.restype = ctypes.c_int
     lib.onnx_conv2d_add_run.argtypes = [vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.onnx_conv2d_prepack.restype = ctypes.c_int
+    lib.onnx_conv2d_prepack.argtypes = [vp, vp, vp, sz, vp]
+    lib.onnx_conv2d_run_prepacked.restype = ctypes.c_int
+    lib.onnx_conv2d_run_prepacked.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.onnx_conv2d_run_static.restype = ctypes.c_int
     lib.onnx_conv2d_run_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.onnx_conv2d_static_scratch_bytes.restype = sz
@@ -197,6 +202,33 @@ class Conv2dDesc:
         _check(self._lib.onnx_conv2d_add_run(self._h, _dev_ptr(X, "X"), _dev_ptr(W, "W"),
                                              _dev_ptr(B, "B", allow_none=True), _dev_ptr(R, "R"), _dev_ptr(Y, "Y"),
                                              ws_ptr, ws_len, _stream_ptr(stream)), "onnx_conv2d_add_run")
+        return Y
+
+    def prepack(self, W, stream=None):
+        """``onnx_conv2d_prepack``: the packed copy of constant weights (a uint8 device tensor; empty when
+        this descriptor's kernel reads W directly)."""
+        import torch
+        packed = torch.empty(max(self.workspace_bytes, 16) if self.kernel_family == "mma_implicit" else 16,
+                             dtype=torch.uint8, device=W.device)
+        _check(self._lib.onnx_conv2d_prepack(self._h, _dev_ptr(W, "W"), ctypes.c_void_p(packed.data_ptr()),
+                                             packed.numel(), _stream_ptr(stream)), "onnx_conv2d_prepack")
+        return packed
+
+    def run_prepacked(self, X, W, packed, B=None, R=None, Y=None, workspace=None, stream=None):
+        """``onnx_conv2d_run_prepacked``: run (R None) or run_add (R given) from a packed copy of W."""
+        import torch
+        if Y is None:
+            Y = torch.empty(self.y_shape, dtype=torch.float32, device=X.device)
+        needs_ws = self.kernel_family != "mma_implicit" and self.workspace_bytes
+        if workspace is None and needs_ws:
+            workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=X.device)
+        ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+        ws_len = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        _check(self._lib.onnx_conv2d_run_prepacked(self._h, _dev_ptr(X, "X"), _dev_ptr(W, "W"),
+                                                   ctypes.c_void_p(packed.data_ptr()),
+                                                   _dev_ptr(B, "B", allow_none=True), _dev_ptr(R, "R", allow_none=True),
+                                                   _dev_ptr(Y, "Y"), ws_ptr, ws_len, _stream_ptr(stream)),
+               "onnx_conv2d_run_prepacked")
         return Y
 
     def run_static(self, X, W, B=None, Y=None, stream=None):

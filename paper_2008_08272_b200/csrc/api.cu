@@ -105,7 +105,7 @@ static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_
 
 static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const float *W, const float *B,
                                     const float *R, float *Y, void *workspace, size_t workspace_bytes,
-                                    void *cuda_stream) {
+                                    void *cuda_stream, int phase = kTcConvPackAndRun) {
     if (!d || !X || !W || !Y) return ONNXB_ERR_NULL;
     if (misaligned(R)) return ONNXB_ERR_UNSUPPORTED;
     if ((d->g.has_bias != 0) != (B != nullptr)) return ONNXB_ERR_NULL;
@@ -132,7 +132,7 @@ static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const
                                      cuda_stream);
             break;
         case ONNXB_KERNEL_MMA_IMPLICIT:
-            err = launch_tc_conv(d->plan, X, W, B, R, Y, workspace, cuda_stream);
+            err = launch_tc_conv(d->plan, X, W, B, R, Y, workspace, cuda_stream, phase);
             break;
         default:
             return ONNXB_ERR_UNSUPPORTED;
@@ -153,6 +153,29 @@ extern "C" onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t d, const float *
                                             void *cuda_stream) {
     if (!R) return ONNXB_ERR_NULL;
     return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream);
+}
+
+// Weights known ahead of the run (an inference graph's constants, Sec. 3.4.4): the implicit-GEMM
+// kernel's packing step done once, and run calls that take the packed copy instead of redoing it.
+extern "C" onnxb_status onnx_conv2d_prepack(onnxb_conv2d_desc_t d, const float *W, void *packed, size_t packed_bytes,
+                                            void *cuda_stream) {
+    if (!d || !W) return ONNXB_ERR_NULL;
+    if (d->family != ONNXB_KERNEL_MMA_IMPLICIT) return ONNXB_OK;          // the other kernels read W as it is
+    if (!packed || packed_bytes < d->workspace_bytes) return ONNXB_ERR_WORKSPACE;
+    if (misaligned(W) || misaligned(packed)) return ONNXB_ERR_UNSUPPORTED;
+    const int err = launch_tc_conv(d->plan, nullptr, W, nullptr, nullptr, nullptr, packed, cuda_stream, kTcConvPackOnly);
+    return err == 0 ? ONNXB_OK : ONNXB_ERR_CUDA;
+}
+
+extern "C" onnxb_status onnx_conv2d_run_prepacked(onnxb_conv2d_desc_t d, const float *X, const float *W,
+                                                  const void *packed, const float *B, const float *R, float *Y,
+                                                  void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!d) return ONNXB_ERR_NULL;
+    if (d->family != ONNXB_KERNEL_MMA_IMPLICIT)
+        return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream);
+    if (!packed) return ONNXB_ERR_NULL;
+    // the packed copy stands in for the workspace; its size was checked when it was made
+    return conv2d_run_impl(d, X, W, B, R, Y, const_cast<void *>(packed), d->workspace_bytes, cuda_stream, kTcConvRunOnly);
 }
 
 extern "C" size_t onnx_gemm_workspace_bytes(int, int, int64_t, int64_t, int64_t) { return 0; }

@@ -52,8 +52,10 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
 // implicit-GEMM tensor-core convolution (tc_conv.cu)
 bool tc_conv_plan(const ConvGeom &g, TcConvPlan &plan, bool forced = false);
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan);
+// phase: both steps (pack the weights into the workspace, then convolve), or one of them alone
+constexpr int kTcConvPackAndRun = 0, kTcConvPackOnly = 1, kTcConvRunOnly = 2;
 int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, const float *R, float *Y,
-                   void *workspace, void *stream);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
+                   void *workspace, void *stream, int phase = kTcConvPackAndRun);   // 1x1 stride-1 convolution expressible as a batched TMA GEMM
 
 struct GemmProblem {
     int M, N, K;

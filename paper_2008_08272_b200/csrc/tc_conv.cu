@@ -934,14 +934,14 @@ static int max_pairs(size_t smem) {
 size_t tc_conv_workspace_bytes(const TcConvPlan &plan) { return (size_t)plan.packed_floats * 4; }
 
 int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const float *B, const float *R, float *Y,
-                   void *workspace, void *stream) {
+                   void *workspace, void *stream, int phase) {
     using namespace tc_host;
     cudaStream_t st = (cudaStream_t)stream;
     unsigned int *err = device_status_ptr();
     if (!err) return (int)cudaErrorUnknown;
 
-    // 1. pack + round the weights into the workspace
-    {
+    // 1. pack + round the weights into the workspace (skipped when the caller packed them earlier)
+    if (phase != kTcConvRunOnly) {
         const long long vec = plan.packed_floats / 4;
         const int blocks = (int)std::min<long long>((vec + 255) / 256, 148 * 16);
         const cudaError_t e = launch_pdl(pack_weights_kernel, dim3(blocks), dim3(256), 0, st, plan, W,
@@ -949,6 +949,7 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
         count_launch();
         if (e != cudaSuccess) return (int)e;
     }
+    if (phase == kTcConvPackOnly) return 0;
     // 2. the convolution
     CUtensorMap tmX;
     if (plan.raw_mode == 0) {

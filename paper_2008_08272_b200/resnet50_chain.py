@@ -56,12 +56,14 @@ def build_graph(batch: int) -> List[Op]:
 
 
 class Resnet50Chain:
-    def __init__(self, batch: int, device, seed: int = wl.SEED_BASE + 9000):
+    def __init__(self, batch: int, device, seed: int = wl.SEED_BASE + 9000, prepack: bool = True):
         import torch
         self.torch = torch
         self.batch, self.dev = batch, device
         self.ops = build_graph(batch)
         rng = np.random.default_rng(seed)
+        self.prepack = prepack                  # weights are constants of the graph: pack them once (Sec. 3.4.4)
+        self.packed: Dict[str, object] = {}
         self.params: Dict[str, tuple] = {}
         self.descs: Dict[str, binding.Conv2dDesc] = {}
         ws_bytes = 16
@@ -78,6 +80,8 @@ class Resnet50Chain:
                                        fuse_relu=op.relu)
                 self.descs[op.name] = d
                 ws_bytes = max(ws_bytes, d.workspace_bytes)
+                if prepack:
+                    self.packed[op.name] = d.prepack(self.params[op.name][0])
         Wf = rng.standard_normal((2048, 1000), dtype=np.float32) * np.float32(np.sqrt(1.0 / 2048))
         Bf = rng.standard_normal((1000,), dtype=np.float32) * np.float32(0.01)
         self.params["fc"] = (torch.from_numpy(Wf).to(device), torch.from_numpy(Bf).to(device))
@@ -102,7 +106,11 @@ class Resnet50Chain:
         self.buf["input"] = x
         for op in self.ops:
             src, dst = self.buf[op.src], self.buf[op.dst]
-            if op.kind == "conv":
+            if op.kind in ("conv", "conv_add") and self.prepack:
+                W, B = self.params[op.name]
+                R = self.buf[op.res] if op.kind == "conv_add" else None
+                self.descs[op.name].run_prepacked(src, W, self.packed[op.name], B, R, Y=dst, workspace=self.workspace)
+            elif op.kind == "conv":
                 W, B = self.params[op.name]
                 self.descs[op.name].run(src, W, B, Y=dst, workspace=self.workspace)
             elif op.kind == "conv_add":

@@ -408,6 +408,30 @@ def test_conv_add_relu_fused(binding, c, relu):
     assert worst_ratio(Y.cpu().numpy(), want, S) <= 1.0
 
 
+@pytest.mark.parametrize("c", [ADD_CASES[0], ADD_CASES[3], ADD_CASES[4], ADD_CASES[5], ADD_CASES[7]],
+                         ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+@pytest.mark.parametrize("with_r", [False, True])
+def test_conv_prepacked_matches_the_plain_calls(binding, c, with_r):
+    """Packing constant weights once and running from the copy gives bit for bit what the calls that
+    pack at every run give (same kernels, same arithmetic)."""
+    rng = np.random.default_rng(808)
+    dev = torch.device("cuda:0")
+    X = torch.from_numpy(rng.standard_normal(c["x"]).astype(np.float32)).to(dev)
+    W = torch.from_numpy((rng.standard_normal(c["w"]) * 0.1).astype(np.float32)).to(dev)
+    B = torch.from_numpy(rng.standard_normal((c["w"][0],)).astype(np.float32)).to(dev)
+    kw = dict(pads=c.get("pads", (0, 0, 0, 0)), strides=c.get("strides", (1, 1)), group=c.get("group", 1))
+    d = binding.Conv2dDesc(c["x"], c["w"], has_bias=True, fuse_relu=True, **kw)
+    R = torch.from_numpy(rng.standard_normal(d.y_shape).astype(np.float32)).to(dev) if with_r else None
+    want = d.run_add(X, W, B, R) if with_r else d.run(X, W, B)
+    packed = d.prepack(W)
+    got = d.run_prepacked(X, W, packed, B, R)
+    got2 = d.run_prepacked(X, W, packed, B, R)          # the copy is read only: a second run finds it intact
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == 0
+    assert torch.equal(got, want) and torch.equal(got2, want)
+    d.close()
+
+
 def test_tf32_mma_rate_probe(binding):
     """The measurement aid returns a plausible figure: never faster than the tensor pipe's ideal
     n/2 cycles per 128 x n x 8 instruction, and within a factor two of it; bad arguments are refused."""
