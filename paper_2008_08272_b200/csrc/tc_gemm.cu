@@ -42,7 +42,8 @@ constexpr int kEpiWarps = 8;
 constexpr int kABytes = kBM * kBK * 4;             // 16 KB
 constexpr int kStoreBufBytes = 32 * 32 * 4;        // one 32x32 fp32 block
 constexpr int kStagingBytes = kEpiWarps * kStoreBufBytes;   // one block per epilogue warp
-constexpr int kBarrierBytes = 256;
+constexpr int kBarrierBytes = 512;
+constexpr int kResidualBufs = 2;                    // most blocks of the residual addend in flight per epilogue warp
 constexpr int kSmemLimit = 232448;                 // 227 KB opt-in maximum per CTA
 
 #ifdef ONNXB_PROFILE
@@ -70,6 +71,9 @@ struct Params {
     long long c_si, c_sj, c_sb;
     const float *row_bias;     // optional per-row addend (convolution bias)
     const float *R;            // optional addend laid out exactly like Y (a residual connection), added before Relu
+    int r_tma;                 // R is fetched by TMA (when Y is stored by TMA: same geometry), r_bufs blocks ahead
+    int r_bufs;                // 1 or 2 blocks of R in flight per epilogue warp
+    uint32_t staging_bytes;    // Y staging blocks, plus the R blocks when r_tma
     int relu;
     // MN-major B in one copy per stage: a 4-D view (32 columns of a block, K row, block of 32 columns,
     // batch) lets a single box carry all of a tile's 32-column blocks in the order the MMA wants them.
@@ -89,17 +93,19 @@ struct Params {
 template <int kCtas>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmBb, const __grid_constant__ CUtensorMap tmY, const Params p) {
+               const __grid_constant__ CUtensorMap tmBb, const __grid_constant__ CUtensorMap tmY,
+               const __grid_constant__ CUtensorMap tmR, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment by pointer arithmetic on the shared array itself, so that the compiler
     // keeps treating everything derived from it as shared memory (LDS/STS, not generic accesses)
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t *stages = smem;
     uint8_t *staging = smem + (size_t)p.num_stages * p.stage_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + kStagingBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(staging + p.staging_bytes);
     uint64_t *full = bars, *empty = bars + kMaxStages;
     uint64_t *tmem_full = bars + 2 * kMaxStages, *tmem_empty = tmem_full + 2;
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(tmem_empty + 2);
+    uint64_t *r_full = bars + 24;              // [epilogue warp][kResidualBufs]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.tiles_m * p.tiles_n * p.batch;
@@ -116,7 +122,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(&tmem_full[a], 1);
             mbar_init(&tmem_empty[a], kEpiWarps * kCtas);
         }
+        for (int a = 0; a < kEpiWarps * kResidualBufs; ++a) mbar_init(&r_full[a], 1);
         mbar_fence_init();
+        if (p.r_tma) prefetch_tmap(&tmR);
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
         if (p.b_big) prefetch_tmap(&tmBb);
@@ -275,6 +283,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int q = warp & 3;                    // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;          // which half of the tile's 32-column blocks
         uint8_t *buf = staging + (warp - 2) * kStoreBufBytes;
+        // residual blocks fetched by TMA, kResidualBufs in flight per warp (used when p.r_tma)
+        uint8_t *rbuf = staging + kStagingBytes + (warp - 2) * p.r_bufs * kStoreBufBytes;
+        uint64_t *rbar = r_full + (warp - 2) * kResidualBufs;
+        const uint32_t r_mask = (uint32_t)p.r_bufs - 1, r_shift = (uint32_t)p.r_bufs - 1;
+        uint32_t r_issued = 0, r_used = 0;         // blocks requested / consumed so far by this warp
         int acc = 0;
         uint32_t acc_phase = 0;
         GP_DECL;
@@ -283,15 +296,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int tm = t % p.tiles_m;
             const int tn = (t / p.tiles_m) % p.tiles_n;
             const int b = t / (p.tiles_m * p.tiles_n);
+            const int row0 = tm * kBM * kCtas + rank * kBM + q * 32;
+            const int row = row0 + lane;
+            const int nchunk_all = min(p.BN / 32, (p.N - tn * p.BN + 31) / 32);
+            const int c_lo = half ? (nchunk_all + 1) / 2 : 0, c_hi = half ? nchunk_all : (nchunk_all + 1) / 2;
+            // request block `chunk` of R into the next slot of the warp's ring (lane 0; the slot's last
+            // reader finished before the __syncwarp that precedes every call)
+            auto request_r = [&](int chunk) {
+                if (lane == 0) {
+                    const uint32_t slot = r_issued & r_mask;
+                    mbar_arrive_expect_tx(&rbar[slot], kStoreBufBytes);
+                    tma_load_3d(rbuf + slot * kStoreBufBytes, &tmR, &rbar[slot], tn * p.BN + chunk * 32, row0, b);
+                }
+                ++r_issued;
+            };
+            if (p.r_tma && row0 < p.M) {
+                // the tile's first blocks of R travel while the accumulator is still being computed
+                for (int c = c_lo; c < c_hi && c < c_lo + p.r_bufs; ++c) request_r(c);
+            }
             mbar_wait(&tmem_full[acc], acc_phase, p.err, 4);
             tc_fence_after_sync();
             GP_MARK(0);
-            const int row0 = tm * kBM * kCtas + rank * kBM + q * 32;
-            const int row = row0 + lane;
             if (row0 < p.M) {
                 const float rb = (p.row_bias && row < p.M) ? __ldg(p.row_bias + row) : 0.f;
-                const int nchunk_all = min(p.BN / 32, (p.N - tn * p.BN + 31) / 32);
-                const int c_lo = half ? (nchunk_all + 1) / 2 : 0, c_hi = half ? nchunk_all : (nchunk_all + 1) / 2;
                 const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBN);
                 // one 32x32 block: scale, add, activate, hand to the store path
                 auto finish = [&](const uint32_t (&v)[32], int chunk) {
@@ -302,6 +329,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j) {
                             const float x = fmaf(p.alpha, __uint_as_float(v[j]), rb);
                             f[j] = p.relu ? fmaxf(x, 0.f) : x;
+                        }
+                    } else if (p.C == nullptr && p.r_tma) {
+                        // Residual addend by TMA: the block of R lands in the warp's ring with the same 128-byte
+                        // swizzle as the Y staging block, so a lane reads its row back in eight 16-byte pieces;
+                        // the slot is then refilled with the block two ahead.
+                        const uint32_t slot = r_used & r_mask;
+                        mbar_wait(&rbar[slot], (r_used >> r_shift) & 1u, p.err, 6);
+                        ++r_used;
+                        const uint8_t *rb_ = rbuf + slot * kStoreBufBytes;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const float4 t4 = *reinterpret_cast<const float4 *>(rb_ + lane * 128 + ((c ^ (lane & 7)) << 4));
+                            f[4 * c] = fmaf(p.alpha, __uint_as_float(v[4 * c]), rb) + t4.x;
+                            f[4 * c + 1] = fmaf(p.alpha, __uint_as_float(v[4 * c + 1]), rb) + t4.y;
+                            f[4 * c + 2] = fmaf(p.alpha, __uint_as_float(v[4 * c + 2]), rb) + t4.z;
+                            f[4 * c + 3] = fmaf(p.alpha, __uint_as_float(v[4 * c + 3]), rb) + t4.w;
+                        }
+                        __syncwarp();                                             // every lane has read its row
+                        if (chunk + p.r_bufs < c_hi) request_r(chunk + p.r_bufs);
+                        if (p.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.f);
                         }
                     } else if (p.C == nullptr) {
                         // Residual addend R, laid out like Y.  A lane owns a ROW of the block, but rows are
@@ -582,20 +631,25 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     p.num_kb = (g.K + kBK - 1) / kBK;
     p.stage_bytes = (uint32_t)(kABytes + p.BNH * 128);
     p.tx_bytes = p.stage_bytes;
-    int stages = (kSmemLimit - 1024 - kBarrierBytes - kStagingBytes) / (int)p.stage_bytes;
+    p.y_tma = g.y_split == 0 && (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);
+    p.R = g.C ? nullptr : g.residual;
+    p.r_tma = p.R != nullptr && p.y_tma;
+    // two blocks of R per epilogue warp when the operand ring keeps at least three stages beside them
+    p.r_bufs = kResidualBufs;
+    if ((kSmemLimit - 1024 - kBarrierBytes - kStagingBytes * (1 + kResidualBufs)) / (int)p.stage_bytes < 3) p.r_bufs = 1;
+    p.staging_bytes = (uint32_t)(kStagingBytes * (p.r_tma ? 1 + p.r_bufs : 1));
+    int stages = (kSmemLimit - 1024 - kBarrierBytes - (int)p.staging_bytes) / (int)p.stage_bytes;
     p.num_stages = stages > kMaxStages ? kMaxStages : stages;
     p.idesc = tc::make_idesc_tf32(kBM * p.ctas, p.BN, p.a_mn, p.b_mn);
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
     p.row_bias = g.row_bias; p.relu = g.relu;
-    p.R = g.C ? nullptr : g.residual;
     p.Y = g.Y; p.y_ld = g.y_ld; p.y_sb = g.y_bs;
     p.y_split = g.y_split; p.y_group = g.y_group_stride;
-    p.y_tma = g.y_split == 0 && (g.y_ld % 4 == 0) && (g.batch == 1 || g.y_bs % 4 == 0);
     p.err = device_status_ptr();
     if (!p.err) return (int)cudaErrorUnknown;
 
-    CUtensorMap tmA, tmB, tmY;
+    CUtensorMap tmA, tmB, tmY, tmR;
     // operand maps: dim0 is the contiguous axis
     {
         const uint64_t rows = (uint64_t)g.M, k = (uint64_t)g.K;
@@ -642,8 +696,20 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     } else {
         tmY = tmA;   // never dereferenced
     }
+    tmR = tmY;
+    if (p.r_tma) {
+        // the addend has Y's shape and strides, so its view is Y's with another base
+        uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.M, (uint64_t)g.batch};
+        uint64_t str[2] = {(uint64_t)g.y_ld * 4, g.batch > 1 ? (uint64_t)g.y_bs * 4 : (uint64_t)g.y_ld * 4 * g.M};
+        uint32_t box[3] = {32, 32, 1};
+        if ((reinterpret_cast<uintptr_t>(g.residual) & 15) != 0 ||
+            !make_tmap(&tmR, g.residual, 3, dims, str, box, kTmapSwizzle128)) {
+            p.r_tma = 0;                       // plain loads serve an addend that TMA cannot address
+            p.staging_bytes = kStagingBytes;
+        }
+    }
 
-    const size_t smem = 1024 + (size_t)p.num_stages * p.stage_bytes + kStagingBytes + kBarrierBytes;
+    const size_t smem = 1024 + (size_t)p.num_stages * p.stage_bytes + p.staging_bytes + kBarrierBytes;
     const cudaError_t attr_err =
         cudaFuncSetAttribute(p.ctas == 2 ? tc_gemm_kernel<2> : tc_gemm_kernel<1>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
@@ -652,9 +718,9 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     const int grid = (int)(total < units ? total : units) * p.ctas;
     const cudaError_t le =
         p.ctas == 2 ? launch_pdl_cluster(tc_gemm_kernel<2>, 2, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA,
-                                         tmB, tmBb, tmY, p)
+                                         tmB, tmBb, tmY, tmR, p)
                     : launch_pdl(tc_gemm_kernel<1>, dim3(grid), dim3(kThreads), smem, (cudaStream_t)stream, tmA, tmB, tmBb,
-                                 tmY, p);
+                                 tmY, tmR, p);
     count_launch();
     return (int)le;
 }

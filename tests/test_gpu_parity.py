@@ -408,6 +408,35 @@ def test_conv_add_relu_fused(binding, c, relu):
     assert worst_ratio(Y.cpu().numpy(), want, S) <= 1.0
 
 
+def test_conv_add_many_tiles_per_cta(binding):
+    """The fused addend over a launch in which every CTA walks several tiles (the addend's blocks are
+    requested ahead, across tile boundaries): sampled images against the oracle, which treats each
+    image on its own, and the images in between against a second run on those images alone."""
+    rng = np.random.default_rng(9917)
+    n = 40
+    X = rng.standard_normal((n, 64, 56, 56)).astype(np.float32)
+    W = (rng.standard_normal((256, 64, 1, 1)) * np.sqrt(2.0 / 64)).astype(np.float32)
+    B = (rng.standard_normal((256,)) * 0.1).astype(np.float32)
+    R = rng.standard_normal((n, 256, 56, 56)).astype(np.float32)
+    dev = torch.device("cuda:0")
+    d = binding.Conv2dDesc(X.shape, W.shape, has_bias=True, fuse_relu=True)
+    Xd, Wd, Bd, Rd = (torch.from_numpy(a).to(dev) for a in (X, W, B, R))
+    Y = d.run_add(Xd, Wd, Bd, Rd)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == 0
+    d.close()
+    pick = [0, 17, n - 1]
+    conv, S = oracle.conv2d(X[pick], W, B, relu=False)
+    want = np.maximum(conv + R[pick].astype(np.float64), 0.0)
+    assert worst_ratio(Y[pick].cpu().numpy(), want, S) <= 1.0
+    # the same arithmetic on a three-image launch: identical bits image by image
+    d3 = binding.Conv2dDesc(X[pick].shape, W.shape, has_bias=True, fuse_relu=True)
+    Y3 = d3.run_add(Xd[pick].contiguous(), Wd, Bd, Rd[pick].contiguous())
+    torch.cuda.synchronize()
+    d3.close()
+    assert torch.equal(Y3, Y[pick])
+
+
 @pytest.mark.parametrize("c", [ADD_CASES[0], ADD_CASES[3], ADD_CASES[4], ADD_CASES[5], ADD_CASES[7]],
                          ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
 @pytest.mark.parametrize("with_r", [False, True])
