@@ -198,6 +198,42 @@ gather1x1_kernel(const float *__restrict__ X, float *__restrict__ Xg, unsigned t
     }
 }
 
+// Any layout whose pitch is a multiple of four (both layouts have one): four consecutive outputs per
+// thread, indices divided once and then stepped, four independent scalar loads, one 16-byte store.
+__global__ void __launch_bounds__(256)
+gather1x1_quad_kernel(const float *__restrict__ X, float4 *__restrict__ Xg4, unsigned total4, unsigned pitch,
+                      unsigned NPQ, unsigned PQ, unsigned Q, unsigned C, unsigned HW, unsigned rowstep, unsigned sw,
+                      int merged, const ConvDivisor dv_pitch, const ConvDivisor dv_PQ, const ConvDivisor dv_Q) {
+    tc::pdl_launch_dependents();
+    for (unsigned i4 = blockIdx.x * 256u + threadIdx.x; i4 < total4; i4 += gridDim.x * 256u) {
+        const unsigned i = i4 * 4u;
+        const unsigned row = (unsigned)conv_fdiv((int)i, (int)pitch, dv_pitch);   // merged: channel; per image: n*C + c
+        const unsigned j = i - row * pitch;                                        // a multiple of four
+        unsigned n = 0, r = j;
+        if (merged) {
+            n = (unsigned)conv_fdiv((int)j, (int)PQ, dv_PQ);
+            r = j - n * PQ;
+        }
+        unsigned pp = (unsigned)conv_fdiv((int)r, (int)Q, dv_Q), q = r - pp * Q;
+        const float *src[4];
+        bool ok[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const unsigned plane = merged ? n * C + row : row;
+            ok[e] = j + e < NPQ;
+            src[e] = X + (size_t)plane * HW + pp * rowstep + q * sw;
+            // step to the next output pixel: along the row, then to the next row, then to the next image
+            ++r;
+            if (++q == Q) { q = 0; ++pp; }
+            if (r == PQ) { r = 0; pp = 0; q = 0; ++n; }
+        }
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = ok[e] ? gather_round(__ldg(src[e])) : 0.f;
+        Xg4[i4] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+
 // Per-image layout, Q a multiple of 4, W a multiple of 4, column stride 1 or 2: four outputs per
 // thread from one or two aligned 16-byte loads, one 16-byte store.
 template <int SW>
@@ -374,6 +410,15 @@ int launch_gather1x1(const ConvGeom &g, const float *X, float *Xg, long long pit
             gather1x1_vec_kernel<2><<<blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(X),
                                                            reinterpret_cast<float4 *>(Xg), (unsigned)total4, PQ4, Q4,
                                                            HW4, rowstep4);
+    } else if (pitch % 4 == 0) {
+        const long long total4 = total / 4;
+        const unsigned blocks = (unsigned)std::min<long long>((total4 + 255) / 256, 148LL * 32);
+        gather1x1_quad_kernel<<<blocks, 256, 0, st>>>(X, reinterpret_cast<float4 *>(Xg), (unsigned)total4, (unsigned)pitch,
+                                                      (unsigned)(merged ? g.N * g.P * g.Q : g.P * g.Q),
+                                                      (unsigned)(g.P * g.Q), (unsigned)g.Q, (unsigned)g.C,
+                                                      (unsigned)(g.H * g.W), (unsigned)(g.sh * g.W), (unsigned)g.sw,
+                                                      merged ? 1 : 0, conv_divisor((int)pitch), conv_divisor(g.P * g.Q),
+                                                      conv_divisor(g.Q));
     } else {
         const unsigned blocks = (unsigned)std::min<long long>((total + 255) / 256, 148LL * 64);
         gather1x1_kernel<<<blocks, 256, 0, st>>>(X, Xg, (unsigned)total, (unsigned)pitch,
