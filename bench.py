@@ -593,6 +593,71 @@ def run_pool():
     return 0
 
 
+def run_gemm():
+    """ONNX Gemm (Sec. 3.4.3's MatMul + Add target) at a few sizes and attribute sets: device time per
+    launch with L2 flushed before each (ten flush+run pairs minus ten flushes), TFLOP/s against the measured
+    bf16 burst peak x the nominal TF32/bf16 ratio 0.5, and GB/s against the measured copy bandwidth.  One JSON line."""
+    import torch
+    from paper_2008_08272_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    binding.load(build_if_missing=False)
+    peaks = measured_peaks()
+    tf32_peak = peaks["bf16_burst"] * 0.5
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(fn, reps=10):
+        def once(with_run):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(reps):
+                flush.zero_()
+                if with_run:
+                    fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / reps
+        fn()
+        return min(once(True) for _ in range(3)) - min(once(False) for _ in range(3))
+
+    cases = [  # (M, N, K, transA, transB, C shape or None)
+        (64, 1000, 2048, False, True, (1000,)),        # ResNet-50 classifier head, batch 64
+        (1024, 1024, 1024, False, False, None),
+        (4096, 4096, 4096, False, False, (4096,)),
+        (4096, 4096, 4096, False, True, None),
+        (4096, 4096, 4096, True, False, None),
+        (8192, 8192, 8192, False, False, None),
+        (8192, 1024, 512, False, False, (8192, 1)),    # wide output, short reduction: store-bound
+    ]
+    g = torch.Generator(device="cpu").manual_seed(20)
+    out = {"metric": "ONNX Gemm, device time per launch (L2 flushed)", "unit": "us", "dtype": "tf32",
+           "data": "synthetic", "tf32_peak_tflops": tf32_peak,
+           "tf32_peak_source": peaks["source"] + " bf16 burst x nominal tf32/bf16 ratio 0.5",
+           "hbm_peak_gbs": peaks["hbm_gbs"], "ops": {}}
+    for M, N, K, ta, tb, cs in cases:
+        A = torch.randn((K, M) if ta else (M, K), generator=g).to(dev)
+        B = torch.randn((N, K) if tb else (K, N), generator=g).to(dev)
+        C = torch.randn(cs, generator=g).to(dev) if cs else None
+        Y = torch.empty((M, N), device=dev)
+        need = binding.gemm_workspace_bytes(ta, tb, M, N, K)
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+        us = timed(lambda: binding.onnx_gemm(A, B, C, transA=ta, transB=tb, Y=Y, workspace=ws))
+        if binding.last_device_status() != 0:
+            raise SystemExit("device status set during the Gemm sweep")
+        flops = 2.0 * M * N * K
+        nbytes = 4.0 * (M * K + K * N + M * N)
+        name = f"{M}x{N}x{K}" + ("_tA" if ta else "") + ("_tB" if tb else "") + ("_C" + "x".join(map(str, cs)) if cs else "")
+        out["ops"][name] = {"us": round(us, 1), "tflops": round(flops / us / 1e6, 1),
+                            "frac_of_tf32_peak": round(flops / us / 1e6 / tf32_peak, 3),
+                            "gbs": round(nbytes / us / 1e3, 1)}
+        del A, B, C, Y, ws
+    print(json.dumps(out))
+    return 0
+
+
 def measured_clock_max_mhz():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -616,6 +681,8 @@ def main():
     ap.add_argument("--graph", action="store_true", help="with --model: replay the pass from a captured CUDA graph")
     ap.add_argument("--pool", action="store_true",
                     help="time the two pooling operators at ResNet-50 batch-64 sizes instead of the step")
+    ap.add_argument("--gemm", action="store_true",
+                    help="time ONNX Gemm at a few sizes and attribute sets instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
                     help="measure the issue-rate ceiling of the TF32 tensor-core instruction instead of the step")
     args = ap.parse_args()
@@ -626,6 +693,8 @@ def main():
         return run_probe_tf32()
     if args.pool:
         return run_pool()
+    if args.gemm:
+        return run_gemm()
     if args.model:
         return run_model(args)
     return run_ours(args)
