@@ -369,6 +369,7 @@ def test_matmul_add_entry(binding, shape, c_shape):
 ADD_CASES = [
     dict(x=(2, 64, 28, 28), w=(256, 64, 1, 1)),                                   # GEMM, TMA stores, CTA pairs
     dict(x=(3, 96, 14, 14), w=(72, 96, 1, 1)),                                    # GEMM, one CTA per tile
+    dict(x=(11, 64, 56, 56), w=(128, 64, 1, 1)),                                  # GEMM, one CTA, 256-wide tiles: one addend block in flight
     dict(x=(5, 128, 7, 7), w=(320, 128, 1, 1)),                                   # gathered, merged columns
     dict(x=(2, 64, 28, 28), w=(128, 64, 1, 1), strides=(2, 2)),                   # gathered, per image
     dict(x=(2, 32, 30, 30), w=(48, 32, 3, 3), pads=(1, 1, 1, 1)),                 # implicit GEMM
@@ -437,7 +438,7 @@ def test_conv_add_many_tiles_per_cta(binding):
     assert torch.equal(Y3, Y[pick])
 
 
-@pytest.mark.parametrize("c", [ADD_CASES[0], ADD_CASES[3], ADD_CASES[4], ADD_CASES[5], ADD_CASES[7]],
+@pytest.mark.parametrize("c", [ADD_CASES[0], ADD_CASES[4], ADD_CASES[5], ADD_CASES[6], ADD_CASES[8]],
                          ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
 @pytest.mark.parametrize("with_r", [False, True])
 def test_conv_prepacked_matches_the_plain_calls(binding, c, with_r):
