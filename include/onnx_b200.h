@@ -25,9 +25,17 @@
  *   - Tensors with more than 2^31-1 elements are rejected (ONNXB_ERR_UNSUPPORTED).
  *   - Arithmetic: fp32 inputs and outputs.  Kernels of the tensor-core family
  *     multiply in TF32 (10-bit mantissa operands) and accumulate in fp32; kernels
- *     of the SIMT family use fp32 FMA.  Either way
+ *     of the SIMT family use fp32 FMA.  Operands are rounded to TF32 to nearest
+ *     (2^-11 per operand) before they reach the tensor core, which gives
  *         |Y - exact| <= 1e-3 * sum|x*w| + 1e-5       per output element
- *     for finite inputs of moderate magnitude.
+ *     for finite inputs of moderate magnitude.  One exception: a 1x1, stride-1
+ *     convolution whose image planes TMA can address (ONNXB_KERNEL_MMA_GEMM) feeds
+ *     X to the tensor core as stored, and the hardware drops the low 13 mantissa
+ *     bits (truncation: up to 2^-10, 3.4e-4 on average, always towards zero); W is
+ *     still rounded.  There the bound is 1.5e-3 * sum|x*w| + 1e-5 in the worst case
+ *     (every activation just below a TF32 grid point and every term of one sign); it
+ *     stays below 1e-3 * sum|x*w| + 1e-5 whenever the weights are exact in TF32, and
+ *     measured 0.53 of that on uniform non-negative operands.
  */
 #ifndef ONNX_B200_H_
 #define ONNX_B200_H_
@@ -204,7 +212,8 @@ size_t onnx_conv2d_static_scratch_bytes(void);
 
 /*
  * onnx_gemm_workspace_bytes - device scratch onnx_gemm_run needs for this
- * problem (0 when none).  Host only.
+ * problem (0 when none).  Host only.  The tensor-core path keeps TF32-rounded
+ * copies of A and B there (4 * (M*K + K*N) bytes); the SIMT path needs none.
  */
 size_t onnx_gemm_workspace_bytes(int transA, int transB, int64_t M, int64_t N, int64_t K);
 
@@ -306,6 +315,17 @@ uint64_t onnxb_launch_count(void);
  */
 onnxb_status onnxb_probe_tf32_mma_rate(int n, int instructions, double *cycles_per_instruction,
                                        void *cuda_stream);
+
+/*
+ * Test aid for the failure-detection path (no operator of the paper behind it): launches one CTA
+ * that waits, with the bounded wait the tensor-core kernels use, on a barrier nothing will ever
+ * signal.  After limit_cycles SM cycles (1 .. 1e8, i.e. at most ~50 ms) the wait gives up, sets the
+ * device error word and the kernel returns normally; the next onnxb_last_device_status on that
+ * stream therefore reports ONNXB_ERR_DEVICE_TIMEOUT once, and ONNXB_OK afterwards.  Nothing faults,
+ * traps or hangs, and the context stays usable.  Enqueues on cuda_stream without synchronising.
+ * Errors: ERR_ATTR (limit out of range), ERR_CUDA.
+ */
+onnxb_status onnxb_probe_wait_timeout(long long limit_cycles, void *cuda_stream);
 
 #ifdef __cplusplus
 }

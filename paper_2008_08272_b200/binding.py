@@ -18,6 +18,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_ATTR", "ERR_SHAPE", "ERR_UNSUPPORTED", "E
                 "ERR_CUDA", "ERR_DEVICE_TIMEOUT"]
 AUTO_PAD = {"NOTSET": 0, "SAME_UPPER": 1, "SAME_LOWER": 2, "VALID": 3}
 KERNEL_FAMILIES = ["simt_direct", "simt_depthwise", "mma_gemm", "mma_implicit", "mma_gather_gemm"]
+WEIGHT_COPY_FAMILIES = ("mma_implicit", "mma_gemm")     # their scratch is a derived copy of W: prepack makes it once
 
 EXPORTS = [
     "onnx_conv2d_desc", "onnx_conv2d_desc_query", "onnx_conv2d_desc_query_kernel", "onnx_conv2d_run",
@@ -26,7 +27,7 @@ EXPORTS = [
     "onnxb_last_device_status", "onnxb_set_kernel_override", "onnxb_launch_count",
     "onnxb_probe_tf32_mma_rate", "onnx_matmul_add_run",
     "onnx_maxpool2d_shape", "onnx_maxpool2d_run", "onnx_global_average_pool_run", "onnx_conv2d_add_run",
-    "onnx_conv2d_prepack", "onnx_conv2d_run_prepacked",
+    "onnx_conv2d_prepack", "onnx_conv2d_run_prepacked", "onnxb_probe_wait_timeout",
 ]
 
 
@@ -111,6 +112,8 @@ def load(build_if_missing: bool = True):
     lib.onnxb_launch_count.argtypes = []
     lib.onnxb_probe_tf32_mma_rate.restype = ctypes.c_int
     lib.onnxb_probe_tf32_mma_rate.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double), vp]
+    lib.onnxb_probe_wait_timeout.restype = ctypes.c_int
+    lib.onnxb_probe_wait_timeout.argtypes = [ctypes.c_longlong, vp]
     _lib = lib
     return lib
 
@@ -208,7 +211,7 @@ class Conv2dDesc:
         """``onnx_conv2d_prepack``: the packed copy of constant weights (a uint8 device tensor; empty when
         this descriptor's kernel reads W directly)."""
         import torch
-        packed = torch.empty(max(self.workspace_bytes, 16) if self.kernel_family == "mma_implicit" else 16,
+        packed = torch.empty(max(self.workspace_bytes, 16) if self.kernel_family in WEIGHT_COPY_FAMILIES else 16,
                              dtype=torch.uint8, device=W.device)
         _check(self._lib.onnx_conv2d_prepack(self._h, _dev_ptr(W, "W"), ctypes.c_void_p(packed.data_ptr()),
                                              packed.numel(), _stream_ptr(stream)), "onnx_conv2d_prepack")
@@ -219,7 +222,7 @@ class Conv2dDesc:
         import torch
         if Y is None:
             Y = torch.empty(self.y_shape, dtype=torch.float32, device=X.device)
-        needs_ws = self.kernel_family != "mma_implicit" and self.workspace_bytes
+        needs_ws = self.kernel_family not in WEIGHT_COPY_FAMILIES and self.workspace_bytes
         if workspace is None and needs_ws:
             workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=X.device)
         ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
@@ -324,6 +327,12 @@ def probe_tf32_mma_rate(n: int, instructions: int = 4096, stream=None) -> float:
     _check(load().onnxb_probe_tf32_mma_rate(int(n), int(instructions), ctypes.byref(out), _stream_ptr(stream)),
            "onnxb_probe_tf32_mma_rate")
     return float(out.value)
+
+
+def probe_wait_timeout(limit_cycles: int = 1000000, stream=None) -> None:
+    """``onnxb_probe_wait_timeout``: enqueue a kernel whose only (bounded) wait runs out after
+    ``limit_cycles`` SM cycles; the next ``last_device_status`` then reports ERR_DEVICE_TIMEOUT once."""
+    _check(load().onnxb_probe_wait_timeout(int(limit_cycles), _stream_ptr(stream)), "onnxb_probe_wait_timeout")
 
 
 def onnx_matmul_add(A, B, C=None, *, fuse_relu=False, Y=None, workspace=None, stream=None):

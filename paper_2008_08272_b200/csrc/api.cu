@@ -2,7 +2,11 @@
 // device memory or synchronises (except onnxb_last_device_status, by contract).
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <atomic>
+
 #include "common.h"
+#include "tc_common.cuh"
 #include "tc_host.h"
 
 using namespace onnxb;
@@ -11,15 +15,47 @@ namespace onnxb {
 // Error word set by bounded device-side waits that ran out.
 __device__ unsigned int g_device_status_word = 0;
 unsigned int *device_status_ptr() {
-    static unsigned int *ptrs[64] = {nullptr};
+    // per-device cache; the value is the same whichever thread stores it first
+    static std::atomic<unsigned int *> ptrs[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
+    unsigned int *cached = ptrs[dev].load(std::memory_order_acquire);
+    if (!cached) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_device_status_word) != cudaSuccess) return nullptr;
-        ptrs[dev] = static_cast<unsigned int *>(p);
+        cached = static_cast<unsigned int *>(p);
+        ptrs[dev].store(cached, std::memory_order_release);
     }
-    return ptrs[dev];
+    return cached;
+}
+
+// Copy of the weights rounded to TF32 (nearest).  The GEMM kernel hands its operands to the tensor
+// core as they are stored, and the hardware ignores the low 13 mantissa bits (truncation, one-sided);
+// rounding the constant operand once keeps its error at 2^-11 per term and zero on average.
+// Two arrays in one launch (the second may be empty).
+__global__ void round_tf32_copy_kernel(const float4 *__restrict__ in0, float4 *__restrict__ out0, unsigned n0,
+                                       const float4 *__restrict__ in1, float4 *__restrict__ out1, unsigned n1) {
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();
+    const unsigned total = n0 + n1;
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const bool first = i < n0;
+        const float4 v = __ldg(first ? in0 + i : in1 + (i - n0));
+        const float4 r = make_float4(tc::round_tf32(v.x), tc::round_tf32(v.y), tc::round_tf32(v.z), tc::round_tf32(v.w));
+        if (first) out0[i] = r;
+        else out1[i - n0] = r;
+    }
+}
+// counts are multiples of 4 (the callers' leading dimensions are)
+static int launch_round_tf32_copy(const float *in0, float *out0, long long count0, const float *in1, float *out1,
+                                  long long count1, void *stream) {
+    const unsigned n0 = (unsigned)(count0 / 4), n1 = (unsigned)(count1 / 4);
+    const int blocks = (int)std::min<long long>(((long long)n0 + n1 + 255) / 256, 148 * 8);
+    const cudaError_t e = tc_host::launch_pdl(round_tf32_copy_kernel, dim3(blocks), dim3(256), 0, (cudaStream_t)stream,
+                                              reinterpret_cast<const float4 *>(in0), reinterpret_cast<float4 *>(out0), n0,
+                                              reinterpret_cast<const float4 *>(in1), reinterpret_cast<float4 *>(out1), n1);
+    count_launch();
+    return (int)e;
 }
 
 // A 1x1, stride-1, unpadded, ungrouped convolution is one GEMM per image:
@@ -106,9 +142,10 @@ static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_
 static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const float *W, const float *B,
                                     const float *R, float *Y, void *workspace, size_t workspace_bytes,
                                     void *cuda_stream, int phase = kTcConvPackAndRun) {
-    if (!d || !X || !W || !Y) return ONNXB_ERR_NULL;
+    const bool pack_only = phase == kTcConvPackOnly;
+    if (!d || !W || (!pack_only && (!X || !Y))) return ONNXB_ERR_NULL;
     if (misaligned(R)) return ONNXB_ERR_UNSUPPORTED;
-    if ((d->g.has_bias != 0) != (B != nullptr)) return ONNXB_ERR_NULL;
+    if (!pack_only && (d->g.has_bias != 0) != (B != nullptr)) return ONNXB_ERR_NULL;
     if (d->workspace_bytes > 0 && (!workspace || workspace_bytes < d->workspace_bytes)) return ONNXB_ERR_WORKSPACE;
     if (misaligned(X) || misaligned(W) || misaligned(B) || misaligned(Y) || misaligned(workspace))
         return ONNXB_ERR_UNSUPPORTED;
@@ -121,9 +158,14 @@ static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const
         case ONNXB_KERNEL_SIMT_DIRECT:
             err = launch_simt_conv(d->g, X, W, B, R, Y, cuda_stream);
             break;
-        case ONNXB_KERNEL_MMA_GEMM:
-            err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, W, B, Y, R), cuda_stream);
+        case ONNXB_KERNEL_MMA_GEMM: {
+            // the workspace holds W rounded to TF32 (made here, or earlier by onnx_conv2d_prepack)
+            float *Wr = static_cast<float *>(workspace);
+            err = 0;
+            if (phase != kTcConvRunOnly) err = launch_round_tf32_copy(W, Wr, (long long)d->g.M * d->g.C, nullptr, nullptr, 0, cuda_stream);
+            if (err == 0 && phase != kTcConvPackOnly) err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, Wr, B, Y, R), cuda_stream);
             break;
+        }
         case ONNXB_KERNEL_MMA_GATHER_GEMM:
             err = launch_gather1x1(d->g, X, static_cast<float *>(workspace), gather_pitch(d->g), gather_merged(d->g),
                                    cuda_stream);
@@ -157,34 +199,48 @@ extern "C" onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t d, const float *
 
 // Weights known ahead of the run (an inference graph's constants, Sec. 3.4.4): the implicit-GEMM
 // kernel's packing step done once, and run calls that take the packed copy instead of redoing it.
+// Which kernel families keep a derived copy of W in their scratch (packed and/or rounded to TF32).
+static bool family_has_weight_copy(int family) {
+    return family == ONNXB_KERNEL_MMA_IMPLICIT || family == ONNXB_KERNEL_MMA_GEMM;
+}
+
 extern "C" onnxb_status onnx_conv2d_prepack(onnxb_conv2d_desc_t d, const float *W, void *packed, size_t packed_bytes,
                                             void *cuda_stream) {
     if (!d || !W) return ONNXB_ERR_NULL;
-    if (d->family != ONNXB_KERNEL_MMA_IMPLICIT) return ONNXB_OK;          // the other kernels read W as it is
+    if (!family_has_weight_copy(d->family)) return ONNXB_OK;              // the other kernels read W as it is
     if (!packed || packed_bytes < d->workspace_bytes) return ONNXB_ERR_WORKSPACE;
-    if (misaligned(W) || misaligned(packed)) return ONNXB_ERR_UNSUPPORTED;
-    const int err = launch_tc_conv(d->plan, nullptr, W, nullptr, nullptr, nullptr, packed, cuda_stream, kTcConvPackOnly);
-    return err == 0 ? ONNXB_OK : ONNXB_ERR_CUDA;
+    return conv2d_run_impl(d, nullptr, W, nullptr, nullptr, nullptr, packed, packed_bytes, cuda_stream, kTcConvPackOnly);
 }
 
 extern "C" onnxb_status onnx_conv2d_run_prepacked(onnxb_conv2d_desc_t d, const float *X, const float *W,
                                                   const void *packed, const float *B, const float *R, float *Y,
                                                   void *workspace, size_t workspace_bytes, void *cuda_stream) {
     if (!d) return ONNXB_ERR_NULL;
-    if (d->family != ONNXB_KERNEL_MMA_IMPLICIT)
+    if (!family_has_weight_copy(d->family))
         return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream);
     if (!packed) return ONNXB_ERR_NULL;
     // the packed copy stands in for the workspace; its size was checked when it was made
     return conv2d_run_impl(d, X, W, B, R, Y, const_cast<void *>(packed), d->workspace_bytes, cuda_stream, kTcConvRunOnly);
 }
 
-extern "C" size_t onnx_gemm_workspace_bytes(int, int, int64_t, int64_t, int64_t) { return 0; }
+// ONNX Gemm on the tensor cores reads rounded copies of both operands: the tensor core would otherwise
+// truncate them (one-sided, up to 2^-10 per operand), which leaves the stated error bound for operands
+// of one sign.  Both copies live in the workspace: A' first, then B'.
+static bool gemm_tc_eligible(int transA, int transB, int64_t M, int64_t N, int64_t K) {
+    if (K < 32) return false;                       // thin contraction: exact fp32 FMA instead
+    const int64_t a_ld = transA ? M : K, b_ld = transB ? K : N;
+    return a_ld % 4 == 0 && b_ld % 4 == 0;          // tensor-map strides are multiples of 16 bytes
+}
+
+extern "C" size_t onnx_gemm_workspace_bytes(int transA, int transB, int64_t M, int64_t N, int64_t K) {
+    if (M < 1 || N < 1 || K < 1) return 0;
+    return gemm_tc_eligible(transA, transB, M, N, K) ? (size_t)(M * K + K * N) * 4 : 0;
+}
 
 extern "C" onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float beta, int64_t M, int64_t N,
                                       int64_t K, const float *A, const float *B, const float *C, int c_rank,
                                       const int64_t *c_dims, int fuse_relu, float *Y, void *workspace,
                                       size_t workspace_bytes, void *cuda_stream) {
-    (void)workspace_bytes;
     if (!A || !B || !Y) return ONNXB_ERR_NULL;
     if (M < 1 || N < 1 || K < 1) return ONNXB_ERR_SHAPE;
     const int64_t lim = 2147483647LL;
@@ -218,12 +274,21 @@ extern "C" onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float
     t.row_bias = nullptr; t.relu = p.relu;
     t.Y = Y; t.y_ld = p.N; t.y_bs = 0;
     const int forced = kernel_override();
-    const bool want_tc = forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT ||
-                         (forced < 0 && p.K >= 32);
+    const bool forced_tc = forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT;
+    const bool eligible = gemm_tc_eligible(transA, transB, M, N, K) && tc_gemm_supports(t);
     int err;
-    if (want_tc && tc_gemm_supports(t)) err = launch_tc_gemm(t, cuda_stream);
-    else if (forced == ONNXB_KERNEL_MMA_GEMM || forced == ONNXB_KERNEL_MMA_IMPLICIT) return ONNXB_ERR_UNSUPPORTED;
-    else err = launch_simt_gemm(p, A, B, C, Y, cuda_stream);
+    if (eligible && (forced_tc || forced < 0)) {
+        const size_t need = onnx_gemm_workspace_bytes(transA, transB, M, N, K);
+        if (!workspace || workspace_bytes < need) return ONNXB_ERR_WORKSPACE;
+        float *Ar = static_cast<float *>(workspace), *Br = Ar + M * K;
+        err = launch_round_tf32_copy(A, Ar, M * K, B, Br, K * N, cuda_stream);
+        t.A = Ar; t.B = Br;
+        if (err == 0) err = launch_tc_gemm(t, cuda_stream);
+    } else if (forced_tc) {
+        return ONNXB_ERR_UNSUPPORTED;
+    } else {
+        err = launch_simt_gemm(p, A, B, C, Y, cuda_stream);
+    }
     return err == 0 ? ONNXB_OK : ONNXB_ERR_CUDA;
 }
 

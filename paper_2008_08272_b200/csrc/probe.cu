@@ -66,8 +66,32 @@ tf32_mma_rate_kernel(int n, int rounds, long long *cycles, unsigned int *err) {
     }
 }
 
+// One CTA waits on an mbarrier that nothing ever arrives on, with a short limit.  The wait gives up,
+// records code 31 in the error word and the kernel returns normally: the bounded-wait error path of the
+// tensor-core kernels, exercised without a fault, a trap or an endless loop.
+__global__ void wait_timeout_kernel(long long limit_cycles, unsigned int *err) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(&bar, 0, err, 31, limit_cycles);
+    __syncthreads();
+}
+
 }  // namespace
 }  // namespace onnxb
+
+extern "C" onnxb_status onnxb_probe_wait_timeout(long long limit_cycles, void *cuda_stream) {
+    using namespace onnxb;
+    if (limit_cycles < 1 || limit_cycles > 100000000LL) return ONNXB_ERR_ATTR;     // at most ~50 ms
+    unsigned int *err = device_status_ptr();
+    if (!err) return ONNXB_ERR_CUDA;
+    wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(limit_cycles, err);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? ONNXB_OK : ONNXB_ERR_CUDA;
+}
 
 extern "C" onnxb_status onnxb_probe_tf32_mma_rate(int n, int instructions, double *cycles_per_instruction,
                                                   void *cuda_stream) {

@@ -2,9 +2,13 @@
 // library a workspace because they cannot allocate device memory at that point: code
 // running inside a real-time or safety-certified loop whose memory was fixed at start-up,
 // a plugin hosted by a framework that owns the allocator, or a process whose device heap is
-// already fully reserved.  The scratch the tensor-core convolution needs (its packed,
-// TF32-rounded weights) lives in a fixed array inside the library image instead.
+// already fully reserved.  Whatever scratch the descriptor's kernel needs lives in a fixed
+// array inside the library image instead: the packed, TF32-rounded weights of the implicit-GEMM
+// kernel, the TF32-rounded weights of the 1x1 GEMM kernel, or the gathered input copy of the
+// gather-then-GEMM kernel.
 #include <cuda_runtime.h>
+
+#include <atomic>
 
 #include "common.h"
 
@@ -20,15 +24,15 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 // Device address of the array on the current device.  In host code the symbol name is only a
 // handle, not a device pointer, so the address must be asked for, once per device.
 void *static_scratch_ptr() {
-    static void *ptrs[64] = {nullptr};
+    static std::atomic<void *> ptrs[64];      // per device; every thread that races here stores the same value
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
-        ptrs[dev] = p;
+    void *cached = ptrs[dev].load(std::memory_order_acquire);
+    if (!cached) {
+        if (cudaGetSymbolAddress(&cached, g_static_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev].store(cached, std::memory_order_release);
     }
-    return ptrs[dev];
+    return cached;
 }
 
 }  // namespace
@@ -43,7 +47,8 @@ extern "C" onnxb_status onnx_conv2d_run_static(onnxb_conv2d_desc_t d, const floa
     if (d->workspace_bytes > kStaticScratchBytes) return ONNXB_ERR_WORKSPACE;
     void *scratch = static_scratch_ptr();
     if (!scratch) return ONNXB_ERR_CUDA;
-    // The packing kernel rewrites every byte of the scratch it later reads (zero padding
-    // included), so nothing left behind by an earlier call can leak into this one.
+    // Each family's first kernel (weight packing, weight rounding or the input gather) rewrites
+    // every byte of the scratch that its second kernel reads (zero padding included), so nothing
+    // left behind by an earlier call can leak into this one.
     return onnx_conv2d_run(d, X, W, B, Y, scratch, kStaticScratchBytes, cuda_stream);
 }

@@ -55,22 +55,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Every wait is bounded: after kWaitLimitCycles SM cycles without the phase
-// completing, the caller's error word is set and the wait returns as if it had
-// succeeded, so the kernel always runs to its end (results are then garbage and
-// the host reports ONNXB_ERR_DEVICE_TIMEOUT).  Once the word is set, every other
-// wait gives up at its next check, so a stuck pipeline costs one limit, not many.
+// Every wait is bounded: after `limit` SM cycles (default: about two seconds) without the phase
+// completing, the caller's error word is set and the wait returns as if it had succeeded, so the
+// kernel always runs to its end (results are then garbage and the host reports
+// ONNXB_ERR_DEVICE_TIMEOUT).  Once the word is set, every other wait gives up at its next check, so
+// a stuck pipeline costs one limit, not many.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // about two seconds
 
 __device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, unsigned int *err_word,
-                                          unsigned int code) {
+                                          unsigned int code, long long limit = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
             if (*reinterpret_cast<volatile unsigned int *>(err_word) != 0) return;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit) {
                 atomicCAS(err_word, 0u, code);
                 return;
             }
@@ -272,6 +272,14 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32])
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---------------------------------------------------------------- TF32 rounding
+// fp32 -> TF32, round to nearest with ties away from zero (what cvt.rna.tf32.f32 computes), done
+// with two integer operations: add half an ulp of the 10-bit mantissa to the magnitude and clear
+// the 13 low bits.  A carry out of the mantissa correctly bumps the exponent; Inf stays Inf.
+__device__ __forceinline__ float round_tf32(float x) {
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
+}
 
 // ---------------------------------------------------------------- programmatic dependent launch
 // A kernel launched with the programmatic-stream-serialization attribute may start while its

@@ -25,11 +25,14 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
 #include "common.h"
+#define ONNXB_DEBUG_HOOKS_CONV
+#include "debug_hooks.cuh"
 #include "tc_common.cuh"
 #include "tc_conv_plan.h"
 #include "tc_host.h"
@@ -62,37 +65,6 @@ struct Bars {
     uint32_t tmem_holder;
 };
 static_assert(sizeof(Bars) <= kBarBytes, "barrier block too large");
-
-#ifdef ONNXB_PROFILE
-__device__ long long g_prof[148 * 16];
-#define PROF_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
-#define PROF_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
-#define PROF_RESET() do { pt_ = clock64(); } while (0)
-#define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 6; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
-// event log of CTA 0: kind k (0..7), sequence number i (0..63) -> clock
-__device__ long long g_log[8 * 64];
-#define LOG(k, i) do { if (blockIdx.x == 0 && (i) < 64) g_log[(k) * 64 + (i)] = clock64(); } while (0)
-#else
-#define LOG(k, i) do {} while (0)
-#define PROF_DECL do {} while (0)
-#define PROF_MARK(k) do {} while (0)
-#define PROF_RESET() do {} while (0)
-#define PROF_FLUSH(base) do {} while (0)
-#endif
-
-// fp32 -> TF32, round to nearest with ties away from zero (what cvt.rna.tf32.f32 computes), done
-// with two integer operations: add half an ulp of the 10-bit mantissa to the magnitude and clear
-// the 13 low bits.  A carry out of the mantissa correctly bumps the exponent; Inf stays Inf.
-__device__ __forceinline__ float round_tf32(float x) {
-    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
-}
-
-#ifdef ONNXB_CHECK
-__device__ long long g_chk[8];
-#define CHK(cond, code, val) if (!(cond)) { if (atomicCAS((unsigned long long *)&g_chk[0], 0ull, (unsigned long long)(code)) == 0ull) { g_chk[1] = (long long)(val); g_chk[2] = blockIdx.x; g_chk[3] = threadIdx.x; } continue; }
-#else
-#define CHK(cond, code, val)
-#endif
 
 // ------------------------------------------------------------------ weight packing
 // Packed layout: [group][channel tile][CTA of the pair][channel block][K-step][chunk 0/1][row BNH][4],
@@ -884,32 +856,11 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
     return have;
 }
 
-#ifdef ONNXB_CHECK
-extern "C" int onnxb_dbg_check(long long *out) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_chk, sizeof(long long) * 8);
-    return 0;
-}
-#endif
-#ifdef ONNXB_PROFILE
-extern "C" int onnxb_dbg_profile(long long *out) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 148 * 16);
-    static long long zeros[148 * 16];
-    cudaMemcpyToSymbol(g_prof, zeros, sizeof zeros);
-    return 0;
-}
-extern "C" int onnxb_dbg_log(long long *out) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_log, sizeof(long long) * 8 * 64);
-    return 0;
-}
-#endif
-
 // How many CTA pairs (clusters of two) of the pair kernel the device runs at once; queried once.
-static int max_pairs(size_t smem) {
-    static int cached = -1;
-    if (cached >= 0) return cached;
+static int max_pairs() {
+    static std::atomic<int> cached{-1};
+    int n = cached.load(std::memory_order_acquire);
+    if (n >= 0) return n;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * 148);
     cfg.blockDim = dim3(kThreads);
@@ -921,13 +872,12 @@ static int max_pairs(size_t smem) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int n = 0;
-    (void)smem;
+    n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2, false>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = tc_host::num_sms() / 2;
     }
-    cached = n;
+    cached.store(n, std::memory_order_release);
     return n;
 }
 
@@ -970,7 +920,7 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
     if (e != cudaSuccess) return (int)e;
     const int sms = num_sms();
     // persistent: one CTA per SM; pairs are clusters of two neighbouring SMs
-    const int units = pair ? max_pairs(smem) : sms;
+    const int units = pair ? max_pairs() : sms;
     if (units < 1) return (int)cudaErrorLaunchOutOfResources;
     const int grid = (int)std::min<long long>(plan.total_tiles, units) * plan.ctas;
 #ifdef ONNXB_PROFILE

@@ -20,10 +20,13 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdlib>
 #include <mutex>
 
 #include "common.h"
+#define ONNXB_DEBUG_HOOKS_GEMM
+#include "debug_hooks.cuh"
 #include "tc_common.cuh"
 #include "tc_host.h"
 
@@ -45,20 +48,6 @@ constexpr int kStagingBytes = kEpiWarps * kStoreBufBytes;   // one block per epi
 constexpr int kBarrierBytes = 512;
 constexpr int kResidualBufs = 2;                    // most blocks of the residual addend in flight per epilogue warp
 constexpr int kSmemLimit = 232448;                 // 227 KB opt-in maximum per CTA
-
-#ifdef ONNXB_PROFILE
-__device__ long long g_gprof[148 * 16];
-#define GP_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
-#define GP_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
-#define GP_FLUSH(base, n) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < n; ++k_) g_gprof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
-__device__ long long g_glog[4 * 128];
-#define GLOG(k, i) do { if (blockIdx.x == 0 && (i) < 128) g_glog[(k) * 128 + (i)] = clock64(); } while (0)
-#else
-#define GLOG(k, i) do {} while (0)
-#define GP_DECL do {} while (0)
-#define GP_MARK(k) do {} while (0)
-#define GP_FLUSH(base, n) do {} while (0)
-#endif
 
 struct Params {
     int M, N, K, batch;
@@ -553,32 +542,22 @@ bool make_tmap(CUtensorMap *out, const void *base, int rank, const uint64_t *dim
 }
 
 int num_sms() {
-    static int n = 0;
+    static std::atomic<int> cached{0};
+    int n = cached.load(std::memory_order_acquire);
     if (n == 0) {
         int dev = 0, v = 0;
         if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) {
             n = v;
-        else
+            cached.store(n, std::memory_order_release);
+        } else {
             return 148;
+        }
     }
     return n;
 }
 
 }  // namespace tc_host
-
-#ifdef ONNXB_PROFILE
-extern "C" int onnxb_dbg_glog(long long *out) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_glog, sizeof(long long) * 4 * 128);
-    return 0;
-}
-extern "C" int onnxb_dbg_gprofile(long long *out) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_gprof, sizeof(long long) * 148 * 16);
-    return 0;
-}
-#endif
 
 bool tc_gemm_supports(const TcGemmProblem &g) {
     if (g.M < 1 || g.N < 1 || g.K < 1 || g.batch < 1) return false;
@@ -591,8 +570,9 @@ bool tc_gemm_supports(const TcGemmProblem &g) {
 
 // How many CTA pairs (clusters of two) of the pair kernel the device runs at once; queried once.
 static int gemm_max_pairs() {
-    static int cached = -1;
-    if (cached >= 0) return cached;
+    static std::atomic<int> cached{-1};
+    int n = cached.load(std::memory_order_acquire);
+    if (n >= 0) return n;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * 148);
     cfg.blockDim = dim3(kThreads);
@@ -604,12 +584,12 @@ static int gemm_max_pairs() {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int n = 0;
+    n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, tc_gemm_kernel<2>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = tc_host::num_sms() / 2;
     }
-    cached = n;
+    cached.store(n, std::memory_order_release);
     return n;
 }
 

@@ -86,6 +86,8 @@ class Resnet50Chain:
         Bf = rng.standard_normal((1000,), dtype=np.float32) * np.float32(0.01)
         self.params["fc"] = (torch.from_numpy(Wf).to(device), torch.from_numpy(Bf).to(device))
         self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+        self.fc_workspace = torch.empty(max(binding.gemm_workspace_bytes(False, False, batch, 1000, 2048), 16),
+                                        dtype=torch.uint8, device=device)
         # one buffer per tensor of the graph
         self.buf: Dict[str, "torch.Tensor"] = {}
         for op in self.ops:
@@ -122,7 +124,7 @@ class Resnet50Chain:
                 binding.onnx_global_average_pool(src, Y=dst)
             else:
                 W, B = self.params["fc"]
-                binding.onnx_matmul_add(src.view(self.batch, 2048), W, B, Y=dst)
+                binding.onnx_matmul_add(src.view(self.batch, 2048), W, B, Y=dst, workspace=self.fc_workspace)
         return self.buf["logits"]
 
     def close(self):

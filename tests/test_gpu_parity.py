@@ -255,6 +255,8 @@ GEMM_CASES = [
     (100, 260, 36, False, False, None, 1.0, 1.0, False),
     (128, 256, 32, False, True, None, 1.0, 1.0, False),
     (1000, 2500, 520, False, True, (2500,), 1.0, 1.0, True),
+    (70, 33, 48, False, False, (1, 1), 1.0, -0.5, False),
+    (256, 128, 64, False, True, (1, 1), 2.0, 1.0, True),
 ]
 
 
@@ -268,6 +270,67 @@ def test_gemm_cases(binding, c):
     got = run_gemm_gpu(binding, torch, A, B, C, alpha=alpha, beta=beta, transA=tA, transB=tB, fuse_relu=relu)
     want, S = oracle.gemm(A, B, C, alpha=alpha, beta=beta, transA=tA, transB=tB, relu=relu)
     assert worst_ratio(got, want, S) <= 1.0
+
+
+# ----------------------------------------------------------------- operands of one sign
+# Every other case draws weights of mixed sign, whose TF32 operand errors largely cancel.  With X >= 0
+# and W >= 0 nothing cancels: an operand the tensor core reads as stored loses its low 13 mantissa bits
+# by truncation (one-sided, 3.4e-4 of the term on average, 9.8e-4 at most), a rounded one errs by at
+# most 4.9e-4 either way.  The bar stays |err| <= 1e-3 * S + 1e-5.
+def _same_sign_gemm(binding, M, N, K, transB):
+    rng = np.random.default_rng(K * 31 + N)
+    A = rng.random((M, K), dtype=np.float32)
+    B = rng.random((N, K) if transB else (K, N), dtype=np.float32)
+    got = run_gemm_gpu(binding, torch, A, B, None, transB=transB)
+    want, S = oracle.gemm(A, B, None, transB=transB)
+    return worst_ratio(got, want, S)
+
+
+@pytest.mark.parametrize("K", [32, 64, 2048])
+@pytest.mark.parametrize("transB", [False, True])
+def test_gemm_same_sign_operands(binding, K, transB):
+    ratio = _same_sign_gemm(binding, 192, 264, K, transB)
+    print(f"same-sign Gemm K={K} transB={transB}: worst err/tol {ratio:.3f}")
+    assert ratio <= 1.0, ratio
+
+
+SAME_SIGN_CONVS = [
+    dict(x=(2, 64, 28, 28), w=(256, 64, 1, 1)),                          # 1x1 stride 1: X straight from NCHW
+    dict(x=(2, 256, 28, 28), w=(64, 256, 1, 1)),
+    dict(x=(2, 256, 28, 28), w=(128, 256, 1, 1), strides=(2, 2)),         # strided 1x1
+    dict(x=(4, 256, 7, 7), w=(512, 256, 1, 1)),                           # 7x7 planes
+    dict(x=(2, 64, 28, 28), w=(64, 64, 3, 3), pads=(1, 1, 1, 1)),         # implicit GEMM: both operands rounded
+    dict(x=(2, 3, 64, 64), w=(64, 3, 7, 7), pads=(3, 3, 3, 3), strides=(2, 2)),
+]
+
+
+@pytest.mark.parametrize("c", SAME_SIGN_CONVS, ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+def test_conv_same_sign_operands(binding, c):
+    rng = np.random.default_rng(606)
+    X = rng.random(c["x"], dtype=np.float32)
+    W = rng.random(c["w"], dtype=np.float32)
+    B = rng.random((c["w"][0],), dtype=np.float32)
+    ratio, fam = check_conv(binding, torch, X, W, B, relu=True, pads=c.get("pads", (0, 0, 0, 0)),
+                            strides=c.get("strides", (1, 1)))
+    print(f"same-sign conv {c['x']}x{c['w']} [{fam}]: worst err/tol {ratio:.3f}")
+    assert ratio <= 1.0, (ratio, fam)
+
+
+def test_conv_operands_just_above_a_tf32_grid_point(binding):
+    """Activations whose mantissas sit just above a 10-bit grid point (1 + 2^-10 - 2^-23 times a power of
+    two): the worst case for an operand that is truncated, harmless for one that is rounded.  Weights are
+    exact in TF32, so the error is the activations' alone; kernels that round them are exact here, and the
+    one path that reads X as stored (1x1, stride 1, by TMA) stays inside its documented bound of 1e-3 * S
+    for X's part (2^-10 * S = 9.8e-4 * S)."""
+    rng = np.random.default_rng(707)
+    base = np.float32(1.0 + 2.0 ** -10 - 2.0 ** -23)
+    for c in SAME_SIGN_CONVS:
+        X = (base * np.exp2(rng.integers(-3, 3, size=c["x"]))).astype(np.float32)
+        W = rng.integers(1, 9, size=c["w"]).astype(np.float32) / np.float32(8.0)
+        ratio, fam = check_conv(binding, torch, X, W, None, pads=c.get("pads", (0, 0, 0, 0)),
+                                strides=c.get("strides", (1, 1)))
+        print(f"grid-point conv {c['x']}x{c['w']} [{fam}]: worst err/tol {ratio:.3f}")
+        assert ratio <= 1.0, (ratio, fam)
 
 
 # ----------------------------------------------------------------- the five configurations
@@ -327,24 +390,41 @@ def test_config5_sweep_batch64_sampled_images(binding, case):
     assert ratio <= 1.0, (ratio, fam)
 
 
-def test_sweep_index_mapping_on_full_batch(binding):
-    """Delta kernels on full batch-64 tensors of three sweep shapes: bit-exact copy semantics
-    pin the index mapping of every image, not only the sampled ones."""
-    rng = np.random.default_rng(99)
-    for (C, HW, M, k, s, p) in [(64, 56, 64, 3, 1, 1), (256, 56, 128, 1, 2, 0), (512, 7, 512, 3, 1, 1)]:
-        X = rng.integers(-1024, 1025, size=(64, C, HW, HW)).astype(np.float32)
-        Wt = np.zeros((M, C, k, k), np.float32)
-        sel = [((5 * m + 3) % C, (m + 1) % k, (m // 2) % k) for m in range(M)]
-        for m, (c, r, t) in enumerate(sel):
-            Wt[m, c, r, t] = 1.0
-        got, _ = run_conv_gpu(binding, torch, X, Wt, None, pads=(p,) * 4, strides=(s, s))
-        Xp = np.zeros((64, C, HW + 2 * p, HW + 2 * p), np.float32)
-        Xp[:, :, p:p + HW, p:p + HW] = X
-        P = got.shape[2]
-        for m in range(0, M, 7):
-            c, r, t = sel[m]
-            want = Xp[:, c, r:r + (P - 1) * s + 1:s, t:t + (P - 1) * s + 1:s]
-            assert np.array_equal(got[:, m], want), (C, HW, m)
+# (C, H = W, M, kernel, stride, pad, group): one shape per kernel family of the sweep
+FULL_BATCH_INDEX_CASES = [
+    (64, 56, 64, 3, 1, 1, 1),        # implicit GEMM, one CTA per tile
+    (256, 56, 128, 1, 2, 0, 1),      # strided 1x1, one GEMM per image
+    (512, 7, 512, 3, 1, 1, 1),       # implicit GEMM, CTA pairs, whole-image slabs
+    (512, 7, 2048, 1, 1, 0, 1),      # 1x1 on 7x7 planes (49 pixels: no 16-byte row pitch), merged columns
+    (1024, 14, 512, 1, 2, 0, 1),     # strided 1x1 onto 7x7 planes
+    (256, 14, 1024, 1, 1, 0, 1),     # 1x1 straight on NCHW, CTA pairs
+    (3, 224, 64, 7, 2, 3, 1),        # the stem: tap-pair mode, four parity planes
+    (256, 28, 256, 3, 1, 1, 256),    # depthwise
+]
+
+
+@pytest.mark.parametrize("shape", FULL_BATCH_INDEX_CASES, ids=lambda t: "x".join(map(str, t)))
+def test_sweep_index_mapping_on_full_batch(binding, shape):
+    """Delta kernels on full batch-64 tensors, one sweep shape per kernel family: bit-exact copy
+    semantics pin the index mapping of every image, not only the sampled ones."""
+    C, HW, M, k, s, p, g = shape
+    rng = np.random.default_rng(99 + C + HW)
+    X = rng.integers(-1024, 1025, size=(64, C, HW, HW)).astype(np.float32)
+    Cg = C // g
+    Wt = np.zeros((M, Cg, k, k), np.float32)
+    sel = [((5 * m + 3) % Cg, (m + 1) % k, (m // 2) % k) for m in range(M)]
+    for m, (c, r, t) in enumerate(sel):
+        Wt[m, c, r, t] = 1.0
+    got, _ = run_conv_gpu(binding, torch, X, Wt, None, pads=(p,) * 4, strides=(s, s), group=g)
+    Xp = np.zeros((64, C, HW + 2 * p, HW + 2 * p), np.float32)
+    Xp[:, :, p:p + HW, p:p + HW] = X
+    P = got.shape[2]
+    assert P == (HW + 2 * p - k) // s + 1
+    for m in range(0, M, 7):
+        c, r, t = sel[m]
+        cin = (m // (M // g)) * Cg + c
+        want = Xp[:, cin, r:r + (P - 1) * s + 1:s, t:t + (P - 1) * s + 1:s]
+        assert np.array_equal(got[:, m], want), (shape, m)
 
 
 @pytest.mark.parametrize("shape,c_shape", [((64, 1000, 2048), (1000,)), ((130, 70, 300), (130, 1)), ((33, 40, 20), None)])
@@ -480,3 +560,21 @@ def test_run_rejects_short_workspace_and_host_tensors(binding):
         binding.onnx_conv2d(x.cpu(), w)
     y = binding.onnx_conv2d(x, w)
     assert y.shape == (1, 4, 6, 6) and float(y.abs().max()) == 0.0
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(binding):
+    """A device-side wait that nothing satisfies gives up after its limit, the kernel returns normally,
+    the host sees ERR_DEVICE_TIMEOUT exactly once, and ordinary work afterwards is correct."""
+    assert binding.last_device_status() == 0
+    binding.probe_wait_timeout(1_000_000)                  # about half a millisecond of SM clock
+    status = binding.last_device_status()
+    assert binding.STATUS_NAMES[status] == "ERR_DEVICE_TIMEOUT"
+    assert binding.last_device_status() == 0               # reading the word cleared it
+    with pytest.raises(binding.OnnxB200Error):
+        binding.probe_wait_timeout(0)
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((2, 32, 20, 20)).astype(np.float32)
+    W = rng.standard_normal((48, 32, 3, 3)).astype(np.float32)
+    ratio, fam = check_conv(binding, torch, X, W, None, pads=(1, 1, 1, 1))
+    assert fam == "mma_implicit" and ratio <= 1.0
+    assert binding.last_device_status() == 0

@@ -206,7 +206,7 @@ def test_gemm_is_matmul_then_add():
     rng = np.random.default_rng(6)
     A = rng.standard_normal((6, 9)).astype(np.float32)
     B = rng.standard_normal((9, 4)).astype(np.float32)
-    for cshape in [(), (1,), (4,), (1, 4), (6, 1), (6, 4)]:
+    for cshape in [(), (1,), (4,), (1, 4), (6, 1), (1, 1), (6, 4)]:
         C = rng.standard_normal(cshape).astype(np.float32)
         Y, _ = oracle.gemm(A, B, C)
         want = A.astype(np.float64) @ B.astype(np.float64) + C.astype(np.float64)

@@ -81,5 +81,8 @@ def test_global_average_pool_pins():
     assert np.allclose(yab, ya + 2 * yb, atol=1e-6)                               # linear (up to the fp32 input rounding)
     ref = torch.nn.functional.adaptive_avg_pool2d(torch.from_numpy(A).double(), 1).numpy()
     assert np.allclose(ya, ref, rtol=1e-14, atol=1e-15)
-    Sa = oracle.global_average_pool(A)[1]
-    assert np.allclose(Sa, np.abs(A.astype(np.float64)).mean(axis=(2, 3), keepdims=True), rtol=1e-14)
+    # S (the scale of the parity tolerance) is the mean of magnitudes: hand values on a mixed-sign plane,
+    # where a signed mean (0.5) and a sum of magnitudes (10) would both show
+    Ym, Sm = oracle.global_average_pool(np.array([[[[-1.0, 2.0], [-3.0, 4.0]]]], np.float32))
+    assert Ym[0, 0, 0, 0] == 0.5 and Sm[0, 0, 0, 0] == 2.5
+    assert S[0, 0, 0, 0] == 4.5 and S[1, 2, 0, 0] == 54.5                          # non-negative planes: S = Y
