@@ -2,12 +2,22 @@
 """Benchmark: one step = the 53 convolutions of ResNet-50 v1 at batch 64, the
 depthwise case and the classifier-head Gemm, each launched once through the C ABI.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--repack]
 
 Prints ONE JSON line.  `value` is TFLOP/s over the whole step with inputs resident
 in HBM; `e2e` repeats the measurement with host (pinned) inputs copied in and the
 outputs copied back inside the timed region.  `--impl reference` times the fp64
-CPU oracle on a bounded sample of the same workload.
+CPU oracle on a bounded sample of the same workload.  The weights are constants of
+the graph, so their packed / TF32-rounded copies are made once at set-up
+(onnx_conv2d_prepack) and the timed region runs onnx_conv2d_run_prepacked;
+`--repack` times onnx_conv2d_run instead, which redoes that copy at every call.
+With `--gpus N` and no launcher (WORLD_SIZE unset) the script starts its N ranks itself.
+
+    python bench.py --layers [--only SUBSTR] [--repack]
+
+prints one JSON line per distinct layer shape of the step and per configuration 1-4
+(warm and L2-cold device time, TFLOP/s, GB/s, the roofline bound and the fraction of
+it reached), then one summary line.
 """
 from __future__ import annotations
 
@@ -57,6 +67,31 @@ def ncu_traffic(family):
         return None
     return rec["bytes_per_step"] if h.hexdigest() == rec["sha1"] else None
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max clock
+
+
+def tf32_peak_for(peaks, clocks=None, isolated=False):
+    """(TFLOP/s, text): the measured bf16 GEMM rate x the nominal TF32/bf16 ratio 0.5.  The burst figure
+    for launches timed alone or for a region that ran at the maximum SM clock; the sustained one (taken
+    under the power cap) when the clock record shows the region was power-limited."""
+    burst = isolated
+    if not isolated and clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        burst = clocks["sm_mhz"] >= 0.95 * clocks["sm_max_mhz"] and "sw_power_cap" not in clocks.get("reasons", [])
+    key = "bf16_burst" if burst else "bf16_sustained"
+    why = ("launch timed alone" if isolated else "timed region ran at the maximum SM clock, no power cap") if burst \
+        else "timed region under the power cap or below the maximum clock"
+    return peaks[key] * TF32_OVER_BF16, f"{peaks['source']} bf16 {'burst' if burst else 'sustained'} x nominal tf32/bf16 ratio 0.5 ({why})"
+
+
+def roof_of(flops, nbytes, seconds, tensor_peak_tflops, hbm_gbs):
+    """Roofline of one launch or one family: the binding roof, what was achieved against it, the fraction."""
+    t_tensor = flops / (tensor_peak_tflops * 1e12)
+    t_hbm = nbytes / (hbm_gbs * 1e9)
+    if t_tensor >= t_hbm:
+        ach = flops / seconds / 1e12
+        return {"bound": "tensor", "achieved": ach, "peak": tensor_peak_tflops, "unit": "TFLOP/s",
+                "frac": ach / tensor_peak_tflops}
+    ach = nbytes / seconds / 1e9
+    return {"bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s", "frac": ach / hbm_gbs}
 
 
 def step_ops(batch: int = 64):
@@ -224,6 +259,60 @@ def max_over_ranks(value: float, world: int, device=None) -> float:
     return float(t.item())
 
 
+def ranks_reporting(world: int, device=None) -> int:
+    """How many ranks of the job are really there: every rank contributes one to a sum."""
+    if world <= 1:
+        return 1
+    import torch
+    import torch.distributed as dist
+    t = torch.ones(1, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return int(round(float(t.item())))
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU, rendezvous on
+    127.0.0.1), pass rank 0's output through, fail if any rank fails."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env,
+                                      stdout=subprocess.PIPE if r == 0 else subprocess.DEVNULL, text=True))
+    out, _ = procs[0].communicate()
+    codes = [procs[0].returncode] + [p.wait() for p in procs[1:]]
+    sys.stdout.write(out or "")
+    sys.stdout.flush()
+    return 0 if all(c == 0 for c in codes) else 1
+
+
+def run_cpu_dry_run(args):
+    """The rank logic of a multi-GPU run with the kernels left out (gloo on CPU): every rank joins, the
+    slowest rank's time is the job's, rank 0 prints a line whose n_gpus is the number of ranks that
+    reported.  For testing the launch path on a machine without GPUs; the line says what it is."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+    seen = ranks_reporting(world)
+    if seen != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {seen} rank(s) reported")
+    ms = max_over_ranks(10.0 + rank, world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"cpu_dry_run": True, "n_gpus": seen, "ms_per_step": ms, "value": None,
+                          "note": "no kernel ran: launch-path test only"}))
+    return 0
+
+
 def job_tflops(world: int, flops_per_replica_step: float, ms_per_step: float) -> float:
     """Whole-job throughput of `world` independent replicas that each do one step in ms_per_step."""
     return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
@@ -243,6 +332,9 @@ def run_ours(args):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if ranks_reporting(world, dev) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {world} rank(s) are running: launch one rank per GPU "
+                         "(python bench.py --gpus N starts them itself when WORLD_SIZE is unset)")
     binding.load(build_if_missing=False)
 
     convs, gemm = step_ops(args.batch)
@@ -252,7 +344,7 @@ def run_ours(args):
         if not convs:
             raise SystemExit(f"--only {args.only!r} matches no convolution of the step")
     # ---- inputs: seeded host arrays (pinned, reused by the e2e leg) and resident device copies
-    host, devt, descs = [], [], []
+    host, devt, descs, packed = [], [], [], []
     for c in convs:
         X, W, B = wl.conv_inputs(c)
         hx, hw, hb = (torch.from_numpy(t).pin_memory() for t in (X, W, B))
@@ -262,6 +354,7 @@ def run_ours(args):
         ws = torch.empty(max(d.workspace_bytes, 16), dtype=torch.uint8, device=dev)
         y = torch.empty(d.y_shape, dtype=torch.float32, device=dev)
         devt.append([hx.to(dev), hw.to(dev), hb.to(dev), y, ws])
+        packed.append(None if args.repack else d.prepack(devt[-1][1]))
         descs.append(d)
     A, Bm, C = wl.gemm_inputs(gemm)
     g_host = tuple(torch.from_numpy(t).pin_memory() for t in (A, Bm, C))
@@ -278,10 +371,16 @@ def run_ours(args):
     families = [d.kernel_family for d in descs] + ["gemm"]
     n_ops = len(flops_per_op)
 
+    def run_conv(i):
+        x, w, b, y, ws = devt[i]
+        if args.repack:
+            descs[i].run(x, w, b, Y=y, workspace=ws)
+        else:
+            descs[i].run_prepacked(x, w, packed[i], b, None, Y=y, workspace=ws)
+
     def launch_all(events=None):
         for i, d in enumerate(descs):
-            x, w, b, y, ws = devt[i]
-            d.run(x, w, b, Y=y, workspace=ws)
+            run_conv(i)
             if events is not None:
                 events[i + 1].record()
         binding.onnx_gemm(g_dev[0], g_dev[1], g_dev[2], transB=True, Y=g_y, workspace=g_ws)
@@ -336,35 +435,39 @@ def run_ours(args):
         fam_count[f] = fam_count.get(f, 0) + 1
     top = max(fam_time, key=fam_time.get)
     peaks = measured_peaks()
-    tensor_peak = peaks["bf16_sustained"] * TF32_OVER_BF16
-    ach_tflops = fam_flops[top] / (fam_time[top] * 1e-3) / 1e12
-    ach_gbs = fam_bytes[top] / (fam_time[top] * 1e-3) / 1e9
-    if top.startswith("mma"):
-        # a dense contraction fed from HBM: report the roof that binds this family's aggregate
-        t_tensor = fam_flops[top] / (tensor_peak * 1e12)
-        t_hbm = fam_bytes[top] / (peaks["hbm_gbs"] * 1e9)
-        if t_tensor >= t_hbm:
-            roof = {"bound": "tensor", "achieved": ach_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
-                    "frac": ach_tflops / tensor_peak}
+    tensor_peak, tensor_src = tf32_peak_for(peaks, clocks)
+
+    def family_roof(f):
+        secs = fam_time[f] * 1e-3
+        if f.startswith("mma") or f == "gemm":
+            r = roof_of(fam_flops[f], fam_bytes[f], secs, tensor_peak, peaks["hbm_gbs"])
+            r["peak_source"] = tensor_src if r["bound"] == "tensor" else f"{peaks['source']} HBM copy"
+        elif f == "simt_depthwise":
+            gbs = fam_bytes[f] / secs / 1e9
+            r = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                 "frac": gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} HBM copy"}
         else:
-            roof = {"bound": "hbm", "achieved": ach_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": ach_gbs / peaks["hbm_gbs"]}
-        roof["peak_source"] = (f"{peaks['source']} bf16 sustained x nominal tf32/bf16 ratio 0.5"
-                               if roof["bound"] == "tensor" else f"{peaks['source']} HBM copy")
-    elif top == "simt_depthwise":
-        roof = {"bound": "hbm", "achieved": ach_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach_gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} HBM copy"}
-    else:
-        roof = {"bound": "alu", "achieved": ach_tflops, "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s",
-                "frac": ach_tflops / FP32_FMA_PEAK_TFLOPS,
-                "peak_source": "derived: 148 SMs x 128 fp32 FMA/clk x 2 x 1.965 GHz"}
+            tf = fam_flops[f] / secs / 1e12
+            r = {"bound": "alu", "achieved": tf, "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s",
+                 "frac": tf / FP32_FMA_PEAK_TFLOPS,
+                 "peak_source": "derived: 148 SMs x 128 fp32 FMA/clk x 2 x 1.965 GHz"}
+        return r
+
+    roof = family_roof(top)
     only_full = (not args.only) and args.batch == 64
     roof.update({"kernel": top, "launches_per_step": fam_count[top], "ms_per_step": fam_time[top],
                  "basis": "all launches of this kernel family in one step (flops or bytes summed, time summed)",
                  "traffic": ncu_traffic(top) if only_full else None, "traffic_unit": "bytes per step"})
-    families_out = {f: {"ops": fam_count[f], "ms": round(fam_time[f], 4),
-                        "tflops": round(fam_flops[f] / (fam_time[f] * 1e-3) / 1e12, 3),
-                        "gbs": round(fam_bytes[f] / (fam_time[f] * 1e-3) / 1e9, 1)} for f in fam_time}
+    families_out = {}
+    for f in fam_time:
+        r = family_roof(f)
+        families_out[f] = {"ops": fam_count[f], "ms": round(fam_time[f], 4),
+                           "tflops": round(fam_flops[f] / (fam_time[f] * 1e-3) / 1e12, 3),
+                           "gbs": round(fam_bytes[f] / (fam_time[f] * 1e-3) / 1e9, 1),
+                           "bound": r["bound"], "frac": round(r["frac"], 4)}
+    # the step against its own roofline: every op at max(flops / tensor peak, bytes / HBM bandwidth)
+    step_roof_ms = sum(max(fl / (tensor_peak * 1e12), by / (peaks["hbm_gbs"] * 1e9))
+                       for fl, by in zip(flops_per_op, bytes_per_op)) * 1e3
 
     # ---- end to end: pinned host inputs in, results out, every step
     e2e_steps = max(1, min(args.steps, 2))
@@ -402,7 +505,7 @@ def run_ours(args):
     def e2e_step():
         for i, d in enumerate(descs):
             x, w, b, y, ws = devt[i]
-            e2e_op(i, (x, w, b), host[i], lambda: d.run(x, w, b, Y=y, workspace=ws), y)
+            e2e_op(i, (x, w, b), host[i], lambda i=i: run_conv(i), y)
         e2e_op(n_ops - 1, g_dev, g_host,
                lambda: binding.onnx_gemm(g_dev[0], g_dev[1], g_dev[2], transB=True, Y=g_y, workspace=g_ws), g_y)
         first[0] = False
@@ -458,9 +561,14 @@ def run_ours(args):
                    "batch_per_gpu": args.batch, "ops_per_step": n_ops,
                    "gflop_per_step": round(flops_per_step / 1e9, 3),
                    "l2": "inputs larger than L2: every op has its own X/W/Y buffers, ~8 GB touched per step",
+                   "weights": ("re-packed / re-rounded by every run call (--repack)" if args.repack else
+                               "constant weights pre-packed once, outside the timed region (onnx_conv2d_prepack)"),
                    "parallelism": f"replicas x{world} (batch split, no collective)"},
         "pct_of_nominal_tf32_peak_1125": round(100 * value / world / 1125.0, 2),
         "roofline": roof, "kernel_families": families_out,
+        "step_roofline": {"ms": round(step_roof_ms, 4), "frac": round(step_roof_ms / ms_per_step, 4),
+                          "basis": "sum over ops of max(flops / tensor peak, algorithmic bytes / HBM bandwidth)",
+                          "tensor_peak_tflops": tensor_peak, "hbm_gbs": peaks["hbm_gbs"]},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "steps": e2e_steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "pipeline": "copy-in, kernels and read-out on three streams, ordered per op by events"},
@@ -658,6 +766,136 @@ def run_gemm():
     return 0
 
 
+def run_layers(args):
+    """Per-layer measurements: every distinct convolution shape of the step (with its multiplicity), the
+    depthwise case, the head Gemm, and configurations 1-4 at their stated sizes.  For each: device time
+    warm (twenty back-to-back launches between two events) and L2-cold (ten L2-flush + launch pairs minus
+    ten flushes: the event clock ticks every ~2 us), TFLOP/s and algorithmic GB/s of the cold time, the
+    roofline time max(flops / TF32 peak, bytes / HBM bandwidth) and the fraction of it reached.
+    Denominators: MEASURED_PEAKS.json's copy bandwidth, and its bf16 burst GEMM rate x 0.5 (launches
+    timed alone run at the maximum clock).  One JSON line per layer, then a summary line."""
+    import torch
+    from paper_2008_08272_b200 import binding
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    binding.load(build_if_missing=False)
+    peaks = measured_peaks()
+    tensor_peak, tensor_src = tf32_peak_for(peaks, isolated=True)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(fn):
+        def span(n, with_flush, with_run):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n):
+                if with_flush:
+                    flush.zero_()
+                if with_run:
+                    fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / n
+        for _ in range(3):
+            fn()
+        warm = min(span(20, False, True) for _ in range(3))
+        cold = min(span(10, True, True) for _ in range(3)) - min(span(10, True, False) for _ in range(3))
+        return warm, cold
+
+    def emit(name, group, shape, family, mult, flops, nbytes, warm, cold, launches):
+        roof_us = max(flops / (tensor_peak * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9)) * 1e6
+        tiny = flops < 1e8                    # configurations 1 and 2: a few microseconds of launch latency
+        rec = {"layer": name, "group": group, "shape": shape, "family": family, "count_in_step": mult,
+               "launches": launches, "us_warm": round(warm, 2), "us_cold": round(cold, 2),
+               "tflops": round(flops / cold / 1e6, 2), "gbs": round(nbytes / cold / 1e3, 1),
+               "bound": "launch" if tiny else ("tensor" if flops / (tensor_peak * 1e12) >= nbytes / (peaks["hbm_gbs"] * 1e9) else "hbm"),
+               "roofline_us": round(roof_us, 2), "frac": None if tiny else round(roof_us / cold, 3),
+               "gflop": round(flops / 1e9, 3), "mbytes": round(nbytes / 1e6, 2)}
+        print(json.dumps(rec), flush=True)
+        return rec
+
+    def conv_line(c, group, mult):
+        X, W, B = wl.conv_inputs(c)
+        x, w, b = (torch.from_numpy(t).to(dev) for t in (X, W, B))
+        d = binding.Conv2dDesc(c.x_shape, c.w_shape, pads=c.pads, strides=c.strides, dilations=c.dilations,
+                               group=c.group, has_bias=True, fuse_relu=c.relu)
+        ws = torch.empty(max(d.workspace_bytes, 16), dtype=torch.uint8, device=dev)
+        y = torch.empty(d.y_shape, dtype=torch.float32, device=dev)
+        pk = None if args.repack else d.prepack(w)
+        fn = (lambda: d.run(x, w, b, Y=y, workspace=ws)) if args.repack else \
+             (lambda: d.run_prepacked(x, w, pk, b, None, Y=y, workspace=ws))
+        l0 = binding.launch_count()
+        fn()
+        launches = int(binding.launch_count() - l0)
+        warm, cold = timed(fn)
+        if binding.last_device_status() != 0:
+            raise SystemExit(f"device status set while timing {c.name}")
+        rec = emit(c.name, group, {"x": list(c.x_shape), "w": list(c.w_shape), "strides": list(c.strides),
+                                   "pads": list(c.pads), "group": c.group},
+                   d.kernel_family, mult, c.flops, c.algorithmic_bytes, warm, cold, launches)
+        d.close()
+        return rec
+
+    def gemm_line(g, group, mult):
+        A, Bm, C = wl.gemm_inputs(g)
+        a, bm, cc = (torch.from_numpy(t).to(dev) for t in (A, Bm, C))
+        m, n, k = g.mnk
+        y = torch.empty((m, n), dtype=torch.float32, device=dev)
+        ws = torch.empty(max(binding.gemm_workspace_bytes(g.transA, g.transB, m, n, k), 16), dtype=torch.uint8, device=dev)
+        fn = lambda: binding.onnx_gemm(a, bm, cc, alpha=g.alpha, beta=g.beta, transA=g.transA, transB=g.transB,
+                                       fuse_relu=g.relu, Y=y, workspace=ws)
+        l0 = binding.launch_count()
+        fn()
+        launches = int(binding.launch_count() - l0)
+        warm, cold = timed(fn)
+        nbytes = 4 * (m * k + k * n + (int(np.prod(g.c_shape)) if g.c_shape is not None else 0) + m * n)
+        return emit(g.name, group, {"M": m, "N": n, "K": k, "transA": g.transA, "transB": g.transB,
+                                    "c_shape": list(g.c_shape) if g.c_shape is not None else None},
+                    "gemm", mult, g.flops, nbytes, warm, cold, launches)
+
+    convs, head = step_ops(args.batch)
+    seen, order = {}, []
+    for c in convs:
+        key = (c.x_shape, c.w_shape, c.strides, c.pads, c.group)
+        if key in seen:
+            seen[key][1] += 1
+        else:
+            seen[key] = [c, 1]
+            order.append(key)
+    want = lambda name: (not args.only) or any(t in name for t in args.only.split(","))
+    step_us, step_roof = 0.0, 0.0
+    for key in order:
+        c, mult = seen[key]
+        if want(c.name):
+            r = conv_line(c, "step", mult)
+            step_us += r["us_cold"] * mult
+            step_roof += r["roofline_us"] * mult
+    if want(head.name):
+        r = gemm_line(head, "step", 1)
+        step_us += r["us_cold"]
+        step_roof += r["roofline_us"]
+    if args.batch == 64:
+        if want("cfg1"):
+            conv_line(wl.config1_mnist_conv(), "config1", 0)
+        if want("cfg2"):
+            gemm_line(wl.config2_gemm_head(), "config2", 0)
+        if want("cfg3"):
+            conv_line(wl.config3_stage2_3x3(), "config3", 0)
+        for c4 in wl.config4_stem_and_projection():
+            if want(c4.name):
+                conv_line(c4, "config4", 0)
+    print(json.dumps({"summary": "sum over the step's ops of the L2-cold times (count_in_step weighted)",
+                      "us": round(step_us, 1), "roofline_us": round(step_roof, 1),
+                      "frac": round(step_roof / step_us, 3) if step_us else None,
+                      "subset": args.only or None, "batch": args.batch,
+                      "weights": "re-packed every call" if args.repack else "pre-packed once",
+                      "tf32_peak_tflops": tensor_peak, "tf32_peak_source": tensor_src,
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": f"{peaks['source']} HBM copy"}))
+    return 0
+
+
 def measured_clock_max_mhz():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -685,10 +923,22 @@ def main():
                     help="time ONNX Gemm at a few sizes and attribute sets instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
                     help="measure the issue-rate ceiling of the TF32 tensor-core instruction instead of the step")
+    ap.add_argument("--repack", action="store_true",
+                    help="time onnx_conv2d_run (weights re-packed at every call) instead of the pre-packed form")
+    ap.add_argument("--layers", action="store_true",
+                    help="per-layer mode: one JSON line per distinct layer shape of the step and per configuration 1-4")
+    ap.add_argument("--cpu-dry-run", action="store_true",
+                    help="exercise the multi-rank launch path on CPU (gloo), no kernels; for tests")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        return spawn_ranks(args.gpus, sys.argv[1:])
+    if args.cpu_dry_run:
+        return run_cpu_dry_run(args)
     if args.impl == "reference":
         return run_reference(args)
+    if args.layers:
+        return run_layers(args)
     if args.probe_tf32:
         return run_probe_tf32()
     if args.pool:

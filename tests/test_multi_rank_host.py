@@ -72,3 +72,23 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(out0.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` with no RANK / WORLD_SIZE in the environment starts two ranks itself;
+    rank 0's line reports the number of ranks that really joined.  (--cpu-dry-run: gloo, no kernels.)"""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--cpu-dry-run"], env=env,
+                          cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=300)
+    assert proc.returncode == 0, proc.stderr
+    line = json.loads(proc.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["cpu_dry_run"] is True
+    assert line["ms_per_step"] == 11.0                 # the slower of the two ranks (10 + rank)
+
+
+def test_bench_refuses_a_rank_count_it_does_not_have():
+    """One process claiming --gpus 2 under a launcher that started only one rank must not print n_gpus 2."""
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--cpu-dry-run"], env=env,
+                          cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, timeout=300)
+    assert proc.returncode != 0 and "n_gpus" not in proc.stdout
