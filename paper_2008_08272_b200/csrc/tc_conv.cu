@@ -6,12 +6,12 @@
 // formed; per block of KB input channels
 //   warp 0      stages the raw NCHW rows the tile touches into shared memory by TMA
 //               (zero fill outside the tensor);
-//   warps 3-10  re-lay them into the K-major "4 channels x slot" operand layout of the MMA,
+//   warps 4-11  re-lay them into the K-major "4 channels x slot" operand layout of the MMA,
 //               rounding fp32 to TF32 (nearest) and writing zeros for padding;
 //   warp 1      streams the pre-packed, pre-rounded weights by bulk copy;
 //   warp 2      issues, for every tap, tcgen05.mma on the SAME activation tile at a start address
 //               shifted by the tap's slot offset, accumulating in TMEM;
-//   warps 11-18 read finished accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
+//   warps 12-19 read finished accumulators back (tcgen05.ld), add bias, apply Relu and store NCHW
 //               with lanes along consecutive pixels (coalesced); when a tile's accumulators fill at
 //               most half of TMEM it holds two sets, so this overlaps the next tile's MMAs.
 // CTA pairs (kCtas = 2): two CTAs of a cluster share one tile of 2 x MT x 128 pixels.  Each stages
@@ -43,10 +43,15 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 608;              // 19 warps: 2 producers, MMA, 8 transform, 8 epilogue
+// Warps: raw producer, weight producer, MMA issuer, 8 transform warps, then kEpi (8 or 4) epilogue warps.
+// With 8 epilogue warps the block has 608 threads and 96 registers per thread; with 4 it has 480 and
+// 128, which the transform warps (ten independent address chains, twenty values in flight) turn into
+// speed: layers bound by the transform and with several tiles per CTA (so that the slower epilogue
+// hides behind the next tile) take the 4-warp form.
 constexpr int kXformWarps = 8;
 constexpr int kXformThreads = kXformWarps * 32;
-constexpr int kEpiWarps = 8;
+constexpr int kFirstXformWarp = 3, kFirstEpiWarp = kFirstXformWarp + kXformWarps;
+constexpr int threads_for(int epi_warps) { return (kFirstEpiWarp + epi_warps) * 32; }
 constexpr int kOwned = 10;                 // (slot, chunk) units of an A stage one transform thread may own
 constexpr int kMaxRawStages = 4;
 constexpr int kMaxAStages = 3;
@@ -110,8 +115,9 @@ __device__ __forceinline__ int cb_rotation(long long tile, int ncb) { return (in
 // ------------------------------------------------------------------ main kernel
 // kAdd: the epilogue also adds a tensor laid out like Y (a residual connection) before the Relu.  A
 // separate instantiation, so that the plain kernel's register allocation is not disturbed.
-template <int kCtas, bool kAdd>
-__global__ void __launch_bounds__(kThreads, 1)
+// kEpiWarps: 8 or 4 epilogue warps (see the thread layout above).
+template <int kCtas, bool kAdd, int kEpiWarps>
+__global__ void __launch_bounds__(threads_for(kEpiWarps), 1)
 tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, const float *__restrict__ X,
                const float *__restrict__ Wpk, const float *__restrict__ bias, const float *__restrict__ R,
                float *__restrict__ Y, unsigned int *err) {
@@ -352,9 +358,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             }
             PROF_FLUSH(0);
         }
-    } else if (warp < 3 + kXformWarps) {
+    } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------ transform warps
-        const int xw = warp - 3;                   // 0..7
+        const int xw = warp - kFirstXformWarp;     // 0..7
         const int xt = xw * 32 + lane;             // 0..255
         const int cp = g.raw_mode == 1 ? g.H * g.W : g.BOXP;    // channel pitch inside the raw stage
         const int per_stage_slots = g.planes * g.SLOTS;
@@ -370,7 +376,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         // What does not depend on the tile is worked out once: where a unit's operand row goes, and
         // which slot of which parity plane it reads.
         uint32_t udst[kOwned];                     // byte offset of the unit's operand row inside an A stage | chunk index
-        uint32_t ujp[kOwned];                      // slot within the plane | plane << 28
+        // plane << 28 | the slot's place in the stage: as slot rows << 12 | slot columns from the tile's first
+        // slot (4 epilogue warps), or as the plain slot index (8)
+        uint32_t ujp[kOwned];
 #pragma unroll
         for (int i = 0; i < kOwned; ++i) {
             udst[i] = 0;
@@ -381,7 +389,11 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 // operand rows are 16 bytes apart: the low four bits carry the unit's chunk index
                 udst[i] = ((uint32_t)ch * (uint32_t)g.chunk_pitch + (uint32_t)idx * 16u) | (uint32_t)ch;
                 const int pl = conv_fdiv(idx, g.SLOTS, g.dv_SLOTS), j = idx - pl * g.SLOTS;
-                ujp[i] = (uint32_t)j | ((uint32_t)pl << 28);
+                // the slot's distance from the tile's first slot, as whole slot rows and columns
+                // (both below 2^12: a stage holds at most kOwned * 256 slots)
+                const int dh = conv_fdiv(j, g.Ws, g.dv_Ws), dw = j - dh * g.Ws;
+                ujp[i] = kEpiWarps == 8 ? (uint32_t)j | ((uint32_t)pl << 28)
+                                        : (uint32_t)dw | ((uint32_t)dh << 12) | ((uint32_t)pl << 28);
             }
         }
         for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
@@ -395,34 +407,72 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 PROF_MARK(4);
                 ++tile_it;
                 const TcConvSegs *segs = reinterpret_cast<const TcConvSegs *>(seg_st + sp * kSegBytes);
+                const int n0 = segs->n_first, hq0 = segs->hq0, wq0 = segs->wq0;
+                if (kEpiWarps == 8) {
+                    // 96 registers per thread: one unit after the other, each leaving early where it can
 #pragma unroll
-                for (int i = 0; i < kOwned; ++i) {
-                    uoff[i] = -1;
-                    if (i < nu) {
-                        const int ch = (int)(udst[i] & 15u), pl = (int)(ujp[i] >> 28);
-                        const uint32_t Gs = (uint32_t)G0 + (ujp[i] & 0x0FFFFFFFu);     // the planner keeps slots below 2^31
-                        if (Gs < (uint32_t)g.total_slots) {
-                            const int n = conv_fdiv((int)Gs, g.L, g.dv_L);
-                            const int uu = (int)Gs - n * g.L;
-                            const int hq = conv_fdiv(uu, g.Ws, g.dv_Ws), wq = uu - hq * g.Ws;
-                            // fixed-index reads of the parity tables (a dynamic index into kernel
-                            // parameters costs an indexed constant load per use)
-                            const int pa = pl == 0 ? g.pa[0] : pl == 1 ? g.pa[1] : pl == 2 ? g.pa[2] : g.pa[3];
-                            const int pb = pl == 0 ? g.pb[0] : pl == 1 ? g.pb[1] : pl == 2 ? g.pb[2] : g.pb[3];
-                            const int h = hq * g.sh + pa - g.pt;
-                            const int w = wq * g.sw + pb - g.pl;
-                            const int sg = n - segs->n_first;
-                            if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
-                                const int f = h * g.W + w - segs->f0[sg];
-                                int o;
-                                if (g.raw_mode == 1) o = segs->base[sg] + f;
-                                else {
-                                    const int bx = conv_fdiv(f, g.BOXP, g.dv_BOXP);
-                                    o = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
+                    for (int i = 0; i < kOwned; ++i) {
+                        uoff[i] = -1;
+                        if (i < nu) {
+                            const int ch = (int)(udst[i] & 15u), pl = (int)(ujp[i] >> 28);
+                            const uint32_t Gs = (uint32_t)G0 + (ujp[i] & 0x0FFFFFFFu);     // the planner keeps slots below 2^31
+                            if (Gs < (uint32_t)g.total_slots) {
+                                const int n = conv_fdiv((int)Gs, g.L, g.dv_L);
+                                const int uu = (int)Gs - n * g.L;
+                                const int hq = conv_fdiv(uu, g.Ws, g.dv_Ws), wq = uu - hq * g.Ws;
+                                // fixed-index reads of the parity tables (a dynamic index into kernel
+                                // parameters costs an indexed constant load per use)
+                                const int pa = pl == 0 ? g.pa[0] : pl == 1 ? g.pa[1] : pl == 2 ? g.pa[2] : g.pa[3];
+                                const int pb = pl == 0 ? g.pb[0] : pl == 1 ? g.pb[1] : pl == 2 ? g.pb[2] : g.pb[3];
+                                const int h = hq * g.sh + pa - g.pt;
+                                const int w = wq * g.sw + pb - g.pl;
+                                const int sg = n - segs->n_first;
+                                if ((unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W && (unsigned)sg < (unsigned)segs->nseg) {
+                                    const int f = h * g.W + w - segs->f0[sg];
+                                    int o;
+                                    if (g.raw_mode == 1) o = segs->base[sg] + f;
+                                    else {
+                                        const int bx = conv_fdiv(f, g.BOXP, g.dv_BOXP);
+                                        o = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
+                                    }
+                                    uoff[i] = o + ch * 4 * cp;
                                 }
-                                uoff[i] = o + ch * 4 * cp;
                             }
                         }
+                    }
+                } else {
+                    // Straight-line code, no branches: the units' chains of dependent integer operations then
+                    // overlap instead of running one after the other (this loop, not the data movement, was
+                    // the larger part of the thin first layer's time when every unit took its own branches).
+                    const int nseg = segs->nseg;
+    #pragma unroll
+                    for (int i = 0; i < kOwned; ++i) {
+                        const int ch = (int)(udst[i] & 15u), pl = (int)(ujp[i] >> 28);
+                        // Slot -> (image, slot row, slot column) without dividing the slot number: the tile's
+                        // first slot was decomposed once (by the producer, in the segment table); this unit
+                        // lies a fixed number of slot rows and columns further on.
+                        int wq = wq0 + (int)(ujp[i] & 0xFFFu);
+                        const int carry = wq >= g.Ws ? 1 : 0;
+                        wq -= carry ? g.Ws : 0;
+                        int hq = hq0 + (int)((ujp[i] >> 12) & 0xFFFu) + carry;
+                        const int k = conv_fdiv(hq, g.Hs, g.dv_Hs);           // images crossed (small images: several)
+                        hq -= k * g.Hs;
+                        // fixed-index reads of the parity tables (a dynamic index into kernel parameters
+                        // costs an indexed constant load per use)
+                        const int pa = pl == 0 ? g.pa[0] : pl == 1 ? g.pa[1] : pl == 2 ? g.pa[2] : g.pa[3];
+                        const int pb = pl == 0 ? g.pb[0] : pl == 1 ? g.pb[1] : pl == 2 ? g.pb[2] : g.pb[3];
+                        const int h = hq * g.sh + pa - g.pt;
+                        const int w = wq * g.sw + pb - g.pl;
+                        const bool ok = i < nu && n0 + k < g.N && (unsigned)h < (unsigned)g.H && (unsigned)w < (unsigned)g.W &&
+                                        k < nseg;
+                        const int sg = k < nseg ? k : 0;                      // a table entry that exists, whatever k is
+                        const int f = h * g.W + w - segs->f0[sg];
+                        int o = segs->base[sg] + f;                           // whole-image slabs
+                        if (g.raw_mode != 1) {
+                            const int bx = g.boxp_shift >= 0 ? (f >> g.boxp_shift) : conv_fdiv(ok ? f : 0, g.BOXP, g.dv_BOXP);
+                            o = segs->base[sg] + bx * box_floats + (f - bx * g.BOXP);
+                        }
+                        uoff[i] = ok ? o + ch * 4 * cp : -1;
                     }
                 }
                 __syncwarp();
@@ -486,9 +536,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
         if (xt == 0) PROF_FLUSH(5);
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int ew = warp - 3 - kXformWarps;     // 0..7
+        const int ew = warp - kFirstEpiWarp;       // 0..7
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
-        const int hf = ew >> 2;
         const long long PQ = (long long)g.P * g.Q;
         const bool two = g.MT == 2;
         const uint32_t acc_empty_addr = kCtas == 2 ? map_to_cta(smem_u32(&bars->acc_empty[0]), 0) : 0u;
@@ -501,6 +550,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             mbar_wait(&bars->acc_full[ab], use & 1u, err, 18);
             tc_fence_after_sync();
             const int nch = (g.BN + 31) / 32;
+            // eight warps: two per TMEM lane quarter, each taking half of the tile; four: one per quarter, both halves
+            for (int hf = ew >> 2; hf < 2; hf += kEpiWarps / 4) {
             int mt, ch_lo, ch_hi;
             if (two) { mt = hf; ch_lo = 0; ch_hi = nch; }
             else { mt = 0; ch_lo = hf ? (nch + 1) / 2 : 0; ch_hi = hf ? nch : (nch + 1) / 2; }
@@ -533,6 +584,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                     if (live) *yp = x;
                     yp += PQ;
                 }
+            }
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -736,6 +788,9 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
         widest = (widest + 3) / 4 * 4;
         const int nbox = (widest + 255) / 256;
         g.BOXP = std::min(256, ((widest + nbox - 1) / nbox + align - 1) / align * align);
+        // Blocks of 4 channels (the thin first layer of a network) stage so little per pixel that whole
+        // 256-pixel boxes cost nothing, and a power of two spares the transform a division per unit.
+        if (g.KB == 4 && widest > 128) g.BOXP = 256;
     }
     {
         int worst = 0;
@@ -775,6 +830,10 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
     g.nb_stages = (int)std::min<long long>(kMaxBStages, room / g.b_stage_bytes);
     g.dv_L = conv_divisor(g.L);
     g.dv_Ws = conv_divisor(g.Ws);
+    g.dv_Hs = conv_divisor(g.Hs);
+    g.boxp_shift = -1;
+    for (int b = 0; b < 16; ++b)
+        if ((1 << b) == g.BOXP) g.boxp_shift = b;
     g.dv_BOXP = conv_divisor(g.BOXP);
     g.dv_SLOTS = conv_divisor(g.SLOTS);
     g.dv_pss = conv_divisor(g.planes * g.SLOTS);
@@ -853,6 +912,16 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
             plan = p;
         }
     }
+    if (have) {
+        // Four epilogue warps (and 128 registers per thread) where the transform paces the kernel and a
+        // CTA walks several tiles: the tap-pair mode of thin first layers (measured: 116 -> 104 us on the
+        // ResNet-50 stem; 16-channel blocks gain nothing).  Pinned by
+        // ONNXB_CONV_EPI = 4 | 8 for A/B measurements.
+        const int units = sms / plan.ctas;
+        plan.epi_warps = (plan.KB == 4 && plan.total_tiles >= 3LL * units) ? 4 : 8;
+        if (const char *e = getenv("ONNXB_CONV_EPI"))
+            if (e[0] == '4' || e[0] == '8') plan.epi_warps = e[0] - '0';
+    }
     return have;
 }
 
@@ -863,7 +932,7 @@ static int max_pairs() {
     if (n >= 0) return n;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * 148);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(threads_for(8));
     cfg.dynamicSmemBytes = kSmemLimit;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -873,7 +942,7 @@ static int max_pairs() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2, false>, &cfg) != cudaSuccess || n < 1) {
+    if (cudaOccupancyMaxActiveClusters(&n, tc_conv_kernel<2, false, 8>, &cfg) != cudaSuccess || n < 1) {
         cudaGetLastError();
         n = tc_host::num_sms() / 2;
     }
@@ -914,8 +983,12 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
                         (size_t)plan.nb_stages * plan.b_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
     const bool pair = plan.ctas == 2;
     const bool add = R != nullptr;
-    auto kern = pair ? (add ? tc_conv_kernel<2, true> : tc_conv_kernel<2, false>)
-                     : (add ? tc_conv_kernel<1, true> : tc_conv_kernel<1, false>);
+    const bool epi4 = plan.epi_warps == 4;
+    auto kern = epi4 ? (pair ? (add ? tc_conv_kernel<2, true, 4> : tc_conv_kernel<2, false, 4>)
+                             : (add ? tc_conv_kernel<1, true, 4> : tc_conv_kernel<1, false, 4>))
+                     : (pair ? (add ? tc_conv_kernel<2, true, 8> : tc_conv_kernel<2, false, 8>)
+                             : (add ? tc_conv_kernel<1, true, 8> : tc_conv_kernel<1, false, 8>));
+    const int threads = threads_for(epi4 ? 4 : 8);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return (int)e;
     const int sms = num_sms();
@@ -930,9 +1003,9 @@ int launch_tc_conv(const TcConvPlan &plan, const float *X, const float *W, const
             plan.raw_stage_bytes, plan.b_stage_bytes, plan.nb_stages, smem);
 #endif
     const cudaError_t le =
-        pair ? launch_pdl_cluster(kern, 2, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+        pair ? launch_pdl_cluster(kern, 2, dim3(grid), dim3(threads), smem, st, tmX, plan, X,
                                   reinterpret_cast<const float *>(workspace), B, R, Y, err)
-             : launch_pdl(kern, dim3(grid), dim3(kThreads), smem, st, tmX, plan, X,
+             : launch_pdl(kern, dim3(grid), dim3(threads), smem, st, tmX, plan, X,
                           reinterpret_cast<const float *>(workspace), B, R, Y, err);
     count_launch();
     return (int)le;

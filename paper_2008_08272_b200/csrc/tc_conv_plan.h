@@ -66,7 +66,9 @@ struct TcConvPlan {
     uint32_t idesc;
     long long packed_floats;         // size of the packed weight buffer
     // divisors device code needs per slot, as multiply-and-shift constants (see conv_fdiv)
-    ConvDivisor dv_L, dv_Ws, dv_BOXP, dv_SLOTS, dv_pss;
+    ConvDivisor dv_L, dv_Ws, dv_Hs, dv_BOXP, dv_SLOTS, dv_pss;
+    int boxp_shift;                  // log2(BOXP) when BOXP is a power of two, else -1
+    int epi_warps;                   // epilogue warps of the launch: 8, or 4 (then 128 registers per thread)
 };
 
 // floor(n / d) for any 32-bit unsigned n.  On the device: the round-up multiply-and-shift method
@@ -97,6 +99,7 @@ inline ConvDivisor conv_divisor(int d) {
 
 struct TcConvSegs {
     int n_first, nseg;
+    int hq0, wq0;                    // slot row / column of the tile's first slot within image n_first
     int f0[kConvMaxSeg];             // first flat pixel (h*W + w) staged for the image
     int base[kConvMaxSeg];           // float offset of the image's data inside the raw stage
     int nbox[kConvMaxSeg];           // boxes (mode 0) / 1 (mode 1) / 0 when nothing of the image is needed
@@ -110,10 +113,16 @@ ONNXB_HD inline void tc_conv_segments(const TcConvPlan &g, long long G0, TcConvS
     if (G0 >= g.total_slots) {       // the second CTA of a pair on the last, half-empty tile
         t.n_first = g.N;
         t.nseg = 0;
+        t.hq0 = t.wq0 = 0;
         t.total_floats = 0;
         return;
     }
     t.n_first = conv_fdiv((int)G0, g.L, g.dv_L);
+    {
+        const int u0 = (int)(G0 - (long long)t.n_first * g.L);
+        t.hq0 = conv_fdiv(u0, g.Ws, g.dv_Ws);
+        t.wq0 = u0 - t.hq0 * g.Ws;
+    }
     const int n_last = conv_fdiv((int)(Gend - 1), g.L, g.dv_L);
     t.nseg = n_last - t.n_first + 1;
     if (t.nseg > kConvMaxSeg) t.nseg = kConvMaxSeg;   // excluded by the planner
