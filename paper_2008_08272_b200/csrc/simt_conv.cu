@@ -259,12 +259,12 @@ gather1x1_vec_kernel(const float4 *__restrict__ X4, float4 *__restrict__ Xg4, un
 
 // Depthwise convolution with unit stride and dilation (group = C = M), the HBM-bound case: 2.25
 // flop per byte, so the only thing that matters is to move each plane once with few instructions.
-// A thread owns a strip of 4 output columns by 2 output rows of one (image, channel) plane, reads
-// the KH + 1 input rows it needs straight from global memory (neighbouring threads' overlapping
-// reads are served by L1) and keeps the window in registers: 21 loads and 72 FMAs for 8 outputs of
-// a 3x3 filter.  VEC: the row pitch and the left pad allow one aligned 16-byte load per row for the
+// A thread owns a strip of 4 output columns by ROWS output rows of one (image, channel) plane, reads
+// the KH + ROWS - 1 input rows it needs straight from global memory (neighbouring threads' overlapping
+// reads are served by L1) and keeps the window in registers: with ROWS = 4 and a 3x3 filter, 18 loads
+// and 144 FMAs for 16 outputs, every input row fetched 1.5 times instead of twice with ROWS = 2.  VEC: the row pitch and the left pad allow one aligned 16-byte load per row for the
 // strip's middle columns; otherwise every column is loaded on its own.
-template <int KH, int KW, bool VEC>
+template <int KH, int KW, bool VEC, int ROWS>
 __global__ void __launch_bounds__(256)
 conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, const float *__restrict__ W,
                              const float *__restrict__ B, const float *__restrict__ R, float *__restrict__ Y,
@@ -272,7 +272,7 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
     constexpr int WIN = KW + 3;                // input columns a strip of 4 outputs touches
     const unsigned i = blockIdx.x * 256u + threadIdx.x;
     if (i >= items) return;
-    // i = (plane * P2 + row pair) * Q4 + column quad; quotients by reciprocal multiplication in
+    // i = (plane * P2 + row group) * Q4 + column quad (P2 = row groups per plane); quotients by reciprocal multiplication in
     // double (right for 31-bit operands up to one unit, which the two comparisons repair)
     unsigned t = __double2uint_rd((double)i * inv_Q4);
     if (t * Q4 > i) --t;
@@ -281,19 +281,23 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
     unsigned plane = __double2uint_rd((double)t * inv_P2);
     if (plane * P2 > t) --plane;
     if ((plane + 1) * P2 <= t) ++plane;
-    const int p0 = (int)(t - plane * P2) * 2, q0 = (int)q4 * 4;
+    const int p0 = (int)(t - plane * P2) * ROWS, q0 = (int)q4 * 4;
     const int c = (int)(plane % (unsigned)g.C);
 
     float w[KH * KW];
 #pragma unroll
     for (int k = 0; k < KH * KW; ++k) w[k] = __ldg(W + (size_t)c * (KH * KW) + k);
     const float bias = B ? __ldg(B + c) : 0.f;
-    float acc0[4] = {bias, bias, bias, bias}, acc1[4] = {bias, bias, bias, bias};
+    float acc[ROWS][4];
+#pragma unroll
+    for (int k = 0; k < ROWS; ++k)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[k][j] = bias;
 
     const float *xp = X + (size_t)plane * g.H * g.W;
     const int iw0 = q0 - g.pl;
 #pragma unroll
-    for (int rr = 0; rr < KH + 1; ++rr) {
+    for (int rr = 0; rr < KH + ROWS - 1; ++rr) {
         const int ih = p0 - g.pt + rr;
         float v[WIN];
 #pragma unroll
@@ -317,20 +321,21 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
                 for (int k = 0; k < WIN; ++k) if ((unsigned)(iw0 + k) < (unsigned)g.W) v[k] = __ldg(row + iw0 + k);
             }
         }
-        // input row rr is filter row rr of output row p0 and filter row rr-1 of output row p0+1
+        // input row rr is filter row rr - k of output row p0 + k
 #pragma unroll
-        for (int s = 0; s < KW; ++s) {
+        for (int k = 0; k < ROWS; ++k) {
+            if (rr - k >= 0 && rr - k < KH) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (rr < KH) acc0[j] = fmaf(v[j + s], w[rr * KW + s], acc0[j]);
-                if (rr >= 1) acc1[j] = fmaf(v[j + s], w[(rr - 1) * KW + s], acc1[j]);
+                for (int s = 0; s < KW; ++s)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[k][j] = fmaf(v[j + s], w[(rr - k) * KW + s], acc[k][j]);
             }
         }
     }
     float *yp = Y + ((size_t)plane * g.P + p0) * g.Q + q0;
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        float *a = k ? acc1 : acc0;
+    for (int k = 0; k < ROWS; ++k) {
+        float *a = acc[k];
         if (p0 + k >= g.P) break;
         if (R) {
             const float *rr = R + (yp - Y) + (size_t)k * g.Q;
@@ -354,18 +359,18 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
 template <int KH, int KW>
 int launch_depthwise_unit(const ConvGeom &g, const float *X, const float *W, const float *B, const float *R, float *Y,
                           cudaStream_t st) {
-    const unsigned Q4 = (unsigned)((g.Q + 3) / 4), P2 = (unsigned)((g.P + 1) / 2);
+    // four output rows per thread where that still gives every SM a few thousand threads, else two
+    const bool rows4 = (long long)g.N * g.C * ((g.P + 3) / 4) * ((g.Q + 3) / 4) >= 148LL * 2048 * 2;
+    const int rows = rows4 ? 4 : 2;
+    const unsigned Q4 = (unsigned)((g.Q + 3) / 4), P2 = (unsigned)((g.P + rows - 1) / rows);
     const long long items = (long long)g.N * g.C * P2 * Q4;
     const unsigned blocks = (unsigned)((items + 255) / 256);
     // aligned 16-byte accesses: every input and output row starts on a 16-byte boundary
     const bool vec = g.pl == 1 && g.W % 4 == 0 && g.Q % 4 == 0 &&
                      (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15) == 0;
-    if (vec)
-        conv2d_depthwise_unit_kernel<KH, KW, true><<<blocks, 256, 0, st>>>(g, X, W, B, R, Y, (unsigned)items, Q4, P2,
-                                                                            1.0 / (double)Q4, 1.0 / (double)P2);
-    else
-        conv2d_depthwise_unit_kernel<KH, KW, false><<<blocks, 256, 0, st>>>(g, X, W, B, R, Y, (unsigned)items, Q4, P2,
-                                                                             1.0 / (double)Q4, 1.0 / (double)P2);
+    auto kern = vec ? (rows4 ? conv2d_depthwise_unit_kernel<KH, KW, true, 4> : conv2d_depthwise_unit_kernel<KH, KW, true, 2>)
+                    : (rows4 ? conv2d_depthwise_unit_kernel<KH, KW, false, 4> : conv2d_depthwise_unit_kernel<KH, KW, false, 2>);
+    kern<<<blocks, 256, 0, st>>>(g, X, W, B, R, Y, (unsigned)items, Q4, P2, 1.0 / (double)Q4, 1.0 / (double)P2);
     count_launch();
     return (int)cudaGetLastError();
 }

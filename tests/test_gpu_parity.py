@@ -182,6 +182,27 @@ def test_conv_implicit_gemm_tile_shapes(binding, c, tile, monkeypatch):
     assert worst_ratio(got, want, S) <= 1.0
 
 
+@pytest.mark.parametrize("c", TILE_CASES + FORCED_IMPLICIT[:4], ids=lambda c: "x".join(map(str, c["x"] + c["w"])))
+def test_conv_implicit_gemm_four_epilogue_warps(binding, c, monkeypatch):
+    """The implicit-GEMM kernel's form with four epilogue warps (the planner picks it for thin first
+    layers only), forced onto ordinary shapes."""
+    rng = np.random.default_rng(404)
+    X = rng.standard_normal(c["x"]).astype(np.float32)
+    W = rng.standard_normal(c["w"]).astype(np.float32)
+    B = rng.standard_normal((c["w"][0],)).astype(np.float32)
+    kw = dict(pads=c.get("pads", (0, 0, 0, 0)), strides=c.get("strides", (1, 1)),
+              dilations=c.get("dilations", (1, 1)), group=c.get("group", 1))
+    monkeypatch.setenv("ONNXB_CONV_EPI", "4")        # read when the descriptor is created
+    binding.set_kernel_override("mma_implicit")
+    try:
+        got, fam = run_conv_gpu(binding, torch, X, W, B, relu=True, **kw)
+    finally:
+        binding.set_kernel_override(None)
+    assert fam == "mma_implicit"
+    want, S = oracle.conv2d(X, W, B, relu=True, **kw)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 @pytest.mark.parametrize("pair", ["0", "1"])
 @pytest.mark.parametrize("shape", [(256, 200, 96), (384, 3136, 64), (300, 260, 130), (512, 64, 1024)])
 def test_gemm_cta_pair_choice(binding, shape, pair, monkeypatch):
