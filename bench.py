@@ -739,6 +739,7 @@ def run_gemm():
         (4096, 4096, 4096, True, False, None),
         (8192, 8192, 8192, False, False, None),
         (8192, 1024, 512, False, False, (8192, 1)),    # wide output, short reduction: store-bound
+        (2048, 2048, 16, False, False, (2048,)),       # thin contraction (K < 32): the exact fp32 SIMT kernel
     ]
     g = torch.Generator(device="cpu").manual_seed(20)
     out = {"metric": "ONNX Gemm, device time per launch (L2 flushed)", "unit": "us", "dtype": "tf32",
