@@ -18,7 +18,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_ATTR", "ERR_SHAPE", "ERR_UNSUPPORTED", "E
                 "ERR_CUDA", "ERR_DEVICE_TIMEOUT"]
 AUTO_PAD = {"NOTSET": 0, "SAME_UPPER": 1, "SAME_LOWER": 2, "VALID": 3}
 KERNEL_FAMILIES = ["simt_direct", "simt_depthwise", "mma_gemm", "mma_implicit", "mma_gather_gemm"]
-WEIGHT_COPY_FAMILIES = ("mma_implicit", "mma_gemm")     # their scratch is a derived copy of W: prepack makes it once
+WEIGHT_COPY_FAMILIES = ("mma_implicit", "mma_gemm", "mma_gather_gemm")   # prepack makes their derived copy of W once
 
 EXPORTS = [
     "onnx_conv2d_desc", "onnx_conv2d_desc_query", "onnx_conv2d_desc_query_kernel", "onnx_conv2d_run",
@@ -222,7 +222,8 @@ class Conv2dDesc:
         import torch
         if Y is None:
             Y = torch.empty(self.y_shape, dtype=torch.float32, device=X.device)
-        needs_ws = self.kernel_family not in WEIGHT_COPY_FAMILIES and self.workspace_bytes
+        needs_ws = (self.kernel_family not in WEIGHT_COPY_FAMILIES or self.kernel_family == "mma_gather_gemm") \
+            and self.workspace_bytes
         if workspace is None and needs_ws:
             workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=X.device)
         ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None

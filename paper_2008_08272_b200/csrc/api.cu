@@ -139,14 +139,19 @@ size_t conv_gather_workspace_bytes(const ConvGeom &g) {
 
 static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
+// w_copy (gather family only): a TF32-rounded copy of W made earlier by onnx_conv2d_prepack; the workspace
+// then only has to hold the gathered input.
 static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const float *W, const float *B,
                                     const float *R, float *Y, void *workspace, size_t workspace_bytes,
-                                    void *cuda_stream, int phase = kTcConvPackAndRun) {
+                                    void *cuda_stream, int phase = kTcConvPackAndRun, const float *w_copy = nullptr) {
     const bool pack_only = phase == kTcConvPackOnly;
     if (!d || !W || (!pack_only && (!X || !Y))) return ONNXB_ERR_NULL;
     if (misaligned(R)) return ONNXB_ERR_UNSUPPORTED;
     if (!pack_only && (d->g.has_bias != 0) != (B != nullptr)) return ONNXB_ERR_NULL;
-    if (d->workspace_bytes > 0 && (!workspace || workspace_bytes < d->workspace_bytes)) return ONNXB_ERR_WORKSPACE;
+    const size_t wr_bytes = (size_t)d->g.M * d->g.C * 4;           // the gather family's rounded weights
+    size_t need = d->workspace_bytes;
+    if (d->family == ONNXB_KERNEL_MMA_GATHER_GEMM) need = pack_only ? wr_bytes : w_copy ? need - wr_bytes : need;
+    if (need > 0 && (!workspace || workspace_bytes < need)) return ONNXB_ERR_WORKSPACE;
     if (misaligned(X) || misaligned(W) || misaligned(B) || misaligned(Y) || misaligned(workspace))
         return ONNXB_ERR_UNSUPPORTED;
 
@@ -166,13 +171,18 @@ static onnxb_status conv2d_run_impl(onnxb_conv2d_desc_t d, const float *X, const
             if (err == 0 && phase != kTcConvPackOnly) err = launch_tc_gemm(conv1x1_as_gemm(d->g, X, Wr, B, Y, R), cuda_stream);
             break;
         }
-        case ONNXB_KERNEL_MMA_GATHER_GEMM:
-            err = launch_gather1x1(d->g, X, static_cast<float *>(workspace), gather_pitch(d->g), gather_merged(d->g),
-                                   cuda_stream);
-            if (err == 0)
-                err = launch_tc_gemm(conv1x1_gathered_as_gemm(d->g, static_cast<const float *>(workspace), W, B, Y, R),
-                                     cuda_stream);
+        case ONNXB_KERNEL_MMA_GATHER_GEMM: {
+            // workspace: [W rounded to TF32][gathered input]; with a copy of W made ahead, the gathered input alone
+            float *ws = static_cast<float *>(workspace);
+            const float *Wr = w_copy ? w_copy : ws;
+            float *Xg = w_copy ? ws : ws + (size_t)d->g.M * d->g.C;
+            err = 0;
+            if (!w_copy) err = launch_round_tf32_copy(W, ws, (long long)d->g.M * d->g.C, nullptr, nullptr, 0, cuda_stream);
+            if (pack_only) break;
+            if (err == 0) err = launch_gather1x1(d->g, X, Xg, gather_pitch(d->g), gather_merged(d->g), cuda_stream);
+            if (err == 0) err = launch_tc_gemm(conv1x1_gathered_as_gemm(d->g, Xg, Wr, B, Y, R), cuda_stream);
             break;
+        }
         case ONNXB_KERNEL_MMA_IMPLICIT:
             err = launch_tc_conv(d->plan, X, W, B, R, Y, workspace, cuda_stream, phase);
             break;
@@ -201,14 +211,16 @@ extern "C" onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t d, const float *
 // kernel's packing step done once, and run calls that take the packed copy instead of redoing it.
 // Which kernel families keep a derived copy of W in their scratch (packed and/or rounded to TF32).
 static bool family_has_weight_copy(int family) {
-    return family == ONNXB_KERNEL_MMA_IMPLICIT || family == ONNXB_KERNEL_MMA_GEMM;
+    return family == ONNXB_KERNEL_MMA_IMPLICIT || family == ONNXB_KERNEL_MMA_GEMM || family == ONNXB_KERNEL_MMA_GATHER_GEMM;
 }
 
 extern "C" onnxb_status onnx_conv2d_prepack(onnxb_conv2d_desc_t d, const float *W, void *packed, size_t packed_bytes,
                                             void *cuda_stream) {
     if (!d || !W) return ONNXB_ERR_NULL;
     if (!family_has_weight_copy(d->family)) return ONNXB_OK;              // the other kernels read W as it is
-    if (!packed || packed_bytes < d->workspace_bytes) return ONNXB_ERR_WORKSPACE;
+    // (the gather family's copy is only the rounded W, the leading part of its workspace)
+    const size_t need = d->family == ONNXB_KERNEL_MMA_GATHER_GEMM ? (size_t)d->g.M * d->g.C * 4 : d->workspace_bytes;
+    if (!packed || packed_bytes < need) return ONNXB_ERR_WORKSPACE;
     return conv2d_run_impl(d, nullptr, W, nullptr, nullptr, nullptr, packed, packed_bytes, cuda_stream, kTcConvPackOnly);
 }
 
@@ -219,6 +231,9 @@ extern "C" onnxb_status onnx_conv2d_run_prepacked(onnxb_conv2d_desc_t d, const f
     if (!family_has_weight_copy(d->family))
         return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream);
     if (!packed) return ONNXB_ERR_NULL;
+    if (d->family == ONNXB_KERNEL_MMA_GATHER_GEMM)      // the copy of W from `packed`, the gathered input in the workspace
+        return conv2d_run_impl(d, X, W, B, R, Y, workspace, workspace_bytes, cuda_stream, kTcConvRunOnly,
+                               static_cast<const float *>(packed));
     // the packed copy stands in for the workspace; its size was checked when it was made
     return conv2d_run_impl(d, X, W, B, R, Y, const_cast<void *>(packed), d->workspace_bytes, cuda_stream, kTcConvRunOnly);
 }

@@ -149,7 +149,7 @@ extern "C" onnxb_status onnx_conv2d_desc(const onnxb_conv2d_attrs *a, onnxb_conv
     }
     d->family = family;
     d->workspace_bytes = family == ONNXB_KERNEL_MMA_IMPLICIT     ? tc_conv_workspace_bytes(d->plan)
-                         : family == ONNXB_KERNEL_MMA_GATHER_GEMM ? conv_gather_workspace_bytes(g)
+                         : family == ONNXB_KERNEL_MMA_GATHER_GEMM ? conv_gather_workspace_bytes(g) + (size_t)g.M * g.C * 4
                          : family == ONNXB_KERNEL_MMA_GEMM        ? (size_t)g.M * g.C * 4      // W rounded to TF32
                                                                   : 0;
     *out = d;
