@@ -522,7 +522,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (kCtas == 2) mbar_arrive_remote(a_full_addr + (uint32_t)as * 8u);   // the issuing CTA's barrier
+                    if (kCtas == 2) mbar_arrive_remote_release(a_full_addr + (uint32_t)as * 8u);   // the issuing CTA's barrier
                     else mbar_arrive(&bars->a_full[as]);
                     mbar_arrive(&bars->raw_empty[rs]);
                 }
