@@ -72,7 +72,7 @@ typedef enum {
     ONNXB_KERNEL_MMA_GEMM = 2,     /* 1x1 stride-1: batched tcgen05 TF32 GEMM straight from NCHW via TMA */
     ONNXB_KERNEL_MMA_IMPLICIT = 3, /* general implicit GEMM: TMA staging + in-smem im2col + tcgen05 TF32 */
     ONNXB_KERNEL_MMA_GATHER_GEMM = 4 /* other 1x1 (strided, or H*W not a multiple of 4): the pixels read are
-                                        gathered into the workspace, then the same batched TF32 GEMM */
+                                        gathered (and rounded) into the workspace, then the same batched TF32 GEMM */
 } onnxb_kernel_family;
 
 /*
@@ -164,15 +164,18 @@ onnxb_status onnx_conv2d_add_run(onnxb_conv2d_desc_t desc, const float *X, const
  * (the usual case in inference; the compiler propagates constants ahead of time, Sec. 3.4.4):
  * the weight re-layout that onnx_conv2d_run performs at every call is done once.
  *
- * onnx_conv2d_prepack writes the packed, TF32-rounded copy of W into `packed` (device, caller-
- * owned, at least the workspace_bytes of onnx_conv2d_desc_query, 16-byte aligned).  Descriptors
- * whose kernel reads W directly need no copy: the call then does nothing and returns OK.
+ * onnx_conv2d_prepack writes the derived copy of W that the descriptor's kernel reads (packed and
+ * rounded to TF32 for ONNXB_KERNEL_MMA_IMPLICIT, rounded to TF32 for ONNXB_KERNEL_MMA_GEMM and
+ * ONNXB_KERNEL_MMA_GATHER_GEMM) into `packed` (device, caller-owned, at least the workspace_bytes
+ * of onnx_conv2d_desc_query, 16-byte aligned).  Descriptors of the SIMT kernels read W directly:
+ * the call then does nothing and returns OK.
  * onnx_conv2d_run_prepacked computes what onnx_conv2d_run (R == NULL) or onnx_conv2d_add_run
- * (R != NULL) computes, from that copy.  W must still be passed (the kernels that use no packed
- * copy read it) and must be the tensor that was packed; `packed` is read only.  workspace /
- * workspace_bytes: as for onnx_conv2d_run for descriptors that use no packed copy, ignored
- * (may be NULL / 0) otherwise.  Errors: as the calls they stand for; ERR_WORKSPACE when `packed`
- * is too small, ERR_NULL when it is missing where needed.
+ * (R != NULL) computes, from that copy, bit for bit.  W must still be passed (the kernels that use
+ * no copy read it) and must be the tensor that was packed; `packed` is read only.  workspace /
+ * workspace_bytes: as for onnx_conv2d_run for the SIMT kernels and for
+ * ONNXB_KERNEL_MMA_GATHER_GEMM (whose gathered input still needs scratch: the queried
+ * workspace_bytes always suffice), ignored (may be NULL / 0) otherwise.  Errors: as the calls they
+ * stand for; ERR_WORKSPACE when `packed` is too small, ERR_NULL when it is missing where needed.
  */
 onnxb_status onnx_conv2d_prepack(onnxb_conv2d_desc_t desc, const float *W, void *packed, size_t packed_bytes,
                                  void *cuda_stream);
