@@ -408,6 +408,7 @@ def test_config5_sweep_batch64_sampled_images(binding, case):
     images 0, 21, 42, 63 exactly (an image's outputs depend on that image only)."""
     X, W, B = wl.conv_inputs(case)
     ratio, fam = check_conv(binding, torch, X, W, B, relu=case.relu, images=[0, 21, 42, 63], **_kw(case))
+    print(f"sweep {case.name} [{fam}]: worst err/tol {ratio:.3f}")
     assert ratio <= 1.0, (ratio, fam)
 
 
