@@ -295,10 +295,15 @@ extern "C" onnxb_status onnx_gemm_run(int transA, int transB, float alpha, float
     if (eligible && (forced_tc || forced < 0)) {
         const size_t need = onnx_gemm_workspace_bytes(transA, transB, M, N, K);
         if (!workspace || workspace_bytes < need) return ONNXB_ERR_WORKSPACE;
-        float *Ar = static_cast<float *>(workspace), *Br = Ar + M * K;
-        err = launch_round_tf32_copy(A, Ar, M * K, B, Br, K * N, cuda_stream);
-        t.A = Ar; t.B = Br;
-        if (err == 0) err = launch_tc_gemm(t, cuda_stream);
+        if (tc_gemm_splitk_fits(t)) {
+            // few tiles and a long reduction: the split-K kernel rounds its operands itself
+            err = launch_tc_gemm(t, cuda_stream);
+        } else {
+            float *Ar = static_cast<float *>(workspace), *Br = Ar + M * K;
+            err = launch_round_tf32_copy(A, Ar, M * K, B, Br, K * N, cuda_stream);
+            t.A = Ar; t.B = Br;
+            if (err == 0) err = launch_tc_gemm(t, cuda_stream);
+        }
     } else if (forced_tc) {
         return ONNXB_ERR_UNSUPPORTED;
     } else {

@@ -595,6 +595,7 @@ static int gemm_max_pairs() {
 
 int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     using namespace tc_host;
+    if (tc_gemm_splitk_fits(g)) return launch_tc_gemm_splitk(g, stream);      // few tiles, long reduction
     Params p{};
     p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
     p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;

@@ -34,6 +34,9 @@ struct TcGemmProblem {
 
 bool tc_gemm_supports(const TcGemmProblem &g);
 int launch_tc_gemm(const TcGemmProblem &g, void *stream);
+// Split-K form for small M and a long reduction (tc_gemm_splitk.cu); launch_tc_gemm uses it where it fits.
+bool tc_gemm_splitk_fits(const TcGemmProblem &g);
+int launch_tc_gemm_splitk(const TcGemmProblem &g, void *stream);
 
 // Address of the device error word of the current device (NULL on failure).
 unsigned int *device_status_ptr();

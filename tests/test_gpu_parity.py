@@ -315,6 +315,30 @@ def test_gemm_same_sign_operands(binding, K, transB):
     assert ratio <= 1.0, ratio
 
 
+@pytest.mark.parametrize("transB", [False, True])
+def test_gemm_same_sign_operands_split_k(binding, transB):
+    """The classifier-head shape takes the split-K kernel, which rounds its operands itself in shared memory."""
+    ratio = _same_sign_gemm(binding, 64, 1000, 2048, transB)
+    print(f"same-sign split-K Gemm 64x1000x2048 transB={transB}: worst err/tol {ratio:.3f}")
+    assert ratio <= 1.0, ratio
+
+
+@pytest.mark.parametrize("shape", ["32,2", "32,4", "64,4", "64,8"])
+@pytest.mark.parametrize("transB", [False, True])
+def test_gemm_split_k_shapes(binding, shape, transB, monkeypatch):
+    """Every tile width and cluster size of the split-K kernel, forced onto a ragged problem (M, N and K
+    no multiples of the tile; the last cluster rank gets a short share of K), with C, alpha, beta and Relu."""
+    monkeypatch.setenv("ONNXB_GEMM_SPLITK", shape)
+    M, N, K = 100, 300, 1000
+    rng = np.random.default_rng(77 + len(shape))
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    B = rng.standard_normal((N, K) if transB else (K, N)).astype(np.float32)
+    C = rng.standard_normal((M, 1)).astype(np.float32)
+    got = run_gemm_gpu(binding, torch, A, B, C, alpha=0.5, beta=-1.5, transB=transB, fuse_relu=True)
+    want, S = oracle.gemm(A, B, C, alpha=0.5, beta=-1.5, transB=transB, relu=True)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 SAME_SIGN_CONVS = [
     dict(x=(2, 64, 28, 28), w=(256, 64, 1, 1)),                          # 1x1 stride 1: X straight from NCHW
     dict(x=(2, 256, 28, 28), w=(64, 256, 1, 1)),
