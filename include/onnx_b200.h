@@ -216,7 +216,9 @@ size_t onnx_conv2d_static_scratch_bytes(void);
 /*
  * onnx_gemm_workspace_bytes - device scratch onnx_gemm_run needs for this
  * problem (0 when none).  Host only.  The tensor-core path keeps TF32-rounded
- * copies of A and B there (4 * (M*K + K*N) bytes); the SIMT path needs none.
+ * copies of A and B there (4 * (M*K + K*N) bytes; its split-K form for small M
+ * rounds in shared memory and leaves the workspace untouched, but the size is
+ * asked for all the same); the SIMT path needs none.
  */
 size_t onnx_gemm_workspace_bytes(int transA, int transB, int64_t M, int64_t N, int64_t K);
 
