@@ -574,6 +574,10 @@ def run_ours(args):
                 "pipeline": "copy-in, kernels and read-out on three streams, ordered per op by events"},
         "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
     }
+    if args.per_op:
+        # every op's own duration inside the step (event after each op), in the step's order
+        names = [c.name for c in convs] + ["head_gemm"]
+        line["per_op_us"] = [[names[i], families[i], round(per_op_ms[i] * 1e3, 1)] for i in range(n_ops)]
     print(json.dumps(line))
     return 0
 
@@ -924,6 +928,8 @@ def main():
                     help="time ONNX Gemm at a few sizes and attribute sets instead of the step")
     ap.add_argument("--probe-tf32", action="store_true",
                     help="measure the issue-rate ceiling of the TF32 tensor-core instruction instead of the step")
+    ap.add_argument("--per-op", action="store_true",
+                    help="add every op's duration inside the step (an event after each op) to the JSON line")
     ap.add_argument("--repack", action="store_true",
                     help="time onnx_conv2d_run (weights re-packed at every call) instead of the pre-packed form")
     ap.add_argument("--layers", action="store_true",

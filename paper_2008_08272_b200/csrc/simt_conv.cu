@@ -296,31 +296,36 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
 
     const float *xp = X + (size_t)plane * g.H * g.W;
     const int iw0 = q0 - g.pl;
+    // Every input row of the window is requested before the first FMA: the kernel is bound by the
+    // latency of these loads, so each thread keeps all of them in flight at once.
+    float v[KH + ROWS - 1][WIN];
 #pragma unroll
     for (int rr = 0; rr < KH + ROWS - 1; ++rr) {
         const int ih = p0 - g.pt + rr;
-        float v[WIN];
 #pragma unroll
-        for (int k = 0; k < WIN; ++k) v[k] = 0.f;
+        for (int k = 0; k < WIN; ++k) v[rr][k] = 0.f;
         if ((unsigned)ih < (unsigned)g.H) {
             const float *row = xp + (size_t)ih * g.W;
             if (VEC) {
                 // pl == 1: columns q0-1 .. q0+KW+1; q0 .. q0+3 are one aligned float4
-                if (iw0 >= 0) v[0] = __ldg(row + iw0);
+                if (iw0 >= 0) v[rr][0] = __ldg(row + iw0);
                 if (q0 + 3 < g.W) {
                     const float4 m = __ldg(reinterpret_cast<const float4 *>(row + q0));
-                    v[1] = m.x; v[2] = m.y; v[3] = m.z; v[4] = m.w;
+                    v[rr][1] = m.x; v[rr][2] = m.y; v[rr][3] = m.z; v[rr][4] = m.w;
                 } else {
 #pragma unroll
-                    for (int k = 1; k < 5; ++k) if (iw0 + k < g.W) v[k] = __ldg(row + iw0 + k);
+                    for (int k = 1; k < 5; ++k) if (iw0 + k < g.W) v[rr][k] = __ldg(row + iw0 + k);
                 }
 #pragma unroll
-                for (int k = 5; k < WIN; ++k) if (iw0 + k < g.W) v[k] = __ldg(row + iw0 + k);
+                for (int k = 5; k < WIN; ++k) if (iw0 + k < g.W) v[rr][k] = __ldg(row + iw0 + k);
             } else {
 #pragma unroll
-                for (int k = 0; k < WIN; ++k) if ((unsigned)(iw0 + k) < (unsigned)g.W) v[k] = __ldg(row + iw0 + k);
+                for (int k = 0; k < WIN; ++k) if ((unsigned)(iw0 + k) < (unsigned)g.W) v[rr][k] = __ldg(row + iw0 + k);
             }
         }
+    }
+#pragma unroll
+    for (int rr = 0; rr < KH + ROWS - 1; ++rr) {
         // input row rr is filter row rr - k of output row p0 + k
 #pragma unroll
         for (int k = 0; k < ROWS; ++k) {
@@ -328,7 +333,7 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
 #pragma unroll
                 for (int s = 0; s < KW; ++s)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) acc[k][j] = fmaf(v[j + s], w[(rr - k) * KW + s], acc[k][j]);
+                    for (int j = 0; j < 4; ++j) acc[k][j] = fmaf(v[rr][j + s], w[(rr - k) * KW + s], acc[k][j]);
             }
         }
     }

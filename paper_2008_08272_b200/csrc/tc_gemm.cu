@@ -55,6 +55,11 @@ struct Params {
     int a_batched, b_batched;
     int BN, tiles_m, tiles_n, num_kb, num_stages;
     uint32_t idesc, stage_bytes, tx_bytes;
+    // The last tile along N is only as wide as the columns left, rounded up to 16: its MMAs take the
+    // descriptor below, and each CTA of a pair stages half of THAT width (so the odd CTA's first column
+    // need not be a multiple of 32, and an MN-major B is then fetched block by block).
+    int nt_tail;               // width of the last tile along N
+    uint32_t idesc_tail;
     float alpha, beta;
     const float *C;            // optional addend, element strides below (0 = broadcast)
     long long c_si, c_sj, c_sb;
@@ -155,9 +160,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int b = t / (p.tiles_m * p.tiles_n);
                 const int ab = p.a_batched ? b : 0, bb = p.b_batched ? b : 0;
                 const int row_a = tm * kBM * kCtas + rank * kBM;        // first A row of this CTA
-                const int col_b = tn * p.BN + rank * p.BNH;             // first B column of this CTA
+                const int bnh_t = (tn == p.tiles_n - 1 ? p.nt_tail : p.BN) / kCtas;     // columns this CTA stages
+                const int col_b = tn * p.BN + rank * bnh_t;             // first B column of this CTA
                 // do all of this CTA's blocks lie among the full ones?  Then one 4-D box brings them.
-                const bool one_box = p.b_mn && p.b_big && col_b / 32 + hb <= p.b_nblk_full;
+                const bool one_box = p.b_mn && p.b_big && (col_b & 31) == 0 && col_b / 32 + hb <= p.b_nblk_full;
+                // block by block: only the blocks the tile needs and that hold columns of B
+                // (never negative: a CTA whose first column lies past N fetches no block at all, and what it
+                // expects on the stage's barrier is exactly what it issues)
+                const int hb_t = col_b < p.N ? min((bnh_t + 31) / 32, (p.N - col_b + 31) / 32) : 0;
+                const uint32_t tx_bytes = (p.b_mn && !one_box) ? (uint32_t)(kABytes + hb_t * 4096) : p.tx_bytes;
                 // This lane's copy.  Every view has four dimensions (the plain ones end in a unit
                 // dimension), so the copies of a stage are ONE instruction executed by several lanes
                 // with their own coordinates; two different copy instructions would run one after the
@@ -178,7 +189,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     c2 = bb;
                     if (!p.b_mn) { active = true; c1 = col_b; d0 = kBK; }
                     else if (one_box) { active = true; tmap = &tmBb; c2 = col_b / 32; c3 = bb; d1 = kBK; }
-                } else if (p.b_mn && !one_box && jb >= 0 && jb < hb) {
+                } else if (p.b_mn && !one_box && jb >= 0 && jb < hb_t) {
                     active = true;
                     tmap = &tmB;
                     dst_off = (uint32_t)kABytes + (uint32_t)jb * 4096u;
@@ -189,7 +200,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
                     if (lane == 0) GLOG(0, glog_i++);
-                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], p.tx_bytes);
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], tx_bytes);
                     __syncwarp();
                     uint8_t *dst = stages + (size_t)stage * p.stage_bytes + dst_off;
                     if (active) tma_load_4d(dst, tmap, &full[stage], c0, c1, c2, c3);
@@ -229,7 +240,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t a_hi = (uint32_t)(a_tmpl >> 32), b_hi = (uint32_t)(b_tmpl >> 32);
             const uint32_t a_lo_c = (uint32_t)a_tmpl, b_lo_c = (uint32_t)b_tmpl;
             const uint32_t a_k16 = (p.a_mn ? 1024u : 32u) >> 4, b_k16 = (p.b_mn ? 1024u : 32u) >> 4;
-            const uint32_t idesc = p.idesc;
             int glog_i = 0, glog_t = 0;
             (void)glog_i; (void)glog_t;
             GP_DECL;
@@ -239,6 +249,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after_sync();
                 GP_MARK(0);
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * kMaxBN;
+                const uint32_t idesc = ((t / p.tiles_m) % p.tiles_n == p.tiles_n - 1) ? p.idesc_tail : p.idesc;
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (kCtas == 2) mbar_wait_cluster(&full[stage], phase, p.err, 3);
                     else mbar_wait(&full[stage], phase, p.err, 3);
@@ -629,6 +640,11 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     int stages = (kSmemLimit - 1024 - kBarrierBytes - (int)p.staging_bytes) / (int)p.stage_bytes;
     p.num_stages = stages > kMaxStages ? kMaxStages : stages;
     p.idesc = tc::make_idesc_tf32(kBM * p.ctas, p.BN, p.a_mn, p.b_mn);
+    {
+        const int left = g.N - (p.tiles_n - 1) * p.BN;
+        p.nt_tail = std::min(p.BN, (left + 15) / 16 * 16);
+        p.idesc_tail = tc::make_idesc_tf32(kBM * p.ctas, p.nt_tail, p.a_mn, p.b_mn);
+    }
     p.alpha = g.alpha; p.beta = g.beta;
     p.C = g.C; p.c_si = g.c_si; p.c_sj = g.c_sj; p.c_sb = g.c_sb;
     p.row_bias = g.row_bias; p.relu = g.relu;

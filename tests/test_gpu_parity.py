@@ -293,6 +293,24 @@ def test_gemm_cases(binding, c):
     assert worst_ratio(got, want, S) <= 1.0
 
 
+@pytest.mark.parametrize("pair", ["0", "1"])
+@pytest.mark.parametrize("transB", [False, True])
+@pytest.mark.parametrize("N", [68, 196, 264, 520, 784, 1028])
+def test_gemm_narrow_last_tile(binding, N, transB, pair, monkeypatch):
+    """The last tile along N is only as wide as the columns left (rounded up to 16), and the two CTAs of a
+    pair split THAT width: 4 columns left (the second CTA then has none), 196 = one narrow tile whose second
+    half starts off a 32-column block, 8 and 16 columns past full tiles, with a ragged K."""
+    monkeypatch.setenv("ONNXB_GEMM_PAIR", pair)
+    M, K = 300, 70
+    rng = np.random.default_rng(N * 7 + int(transB))
+    A = rng.standard_normal((M, K)).astype(np.float32)
+    B = rng.standard_normal((N, K) if transB else (K, N)).astype(np.float32)
+    C = rng.standard_normal((N,)).astype(np.float32)
+    got = run_gemm_gpu(binding, torch, A, B, C, transB=transB, fuse_relu=True)
+    want, S = oracle.gemm(A, B, C, transB=transB, relu=True)
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 # ----------------------------------------------------------------- operands of one sign
 # Every other case draws weights of mixed sign, whose TF32 operand errors largely cancel.  With X >= 0
 # and W >= 0 nothing cancels: an operand the tensor core reads as stored loses its low 13 mantissa bits
