@@ -19,8 +19,9 @@
 // (M = 256) that read both CTAs' shared memory and write each CTA's rows into its own TMEM.  Per
 // CTA this halves the weight bytes fetched from L2 and the weight bytes the tensor pipe reads from
 // shared memory per flop, the two limits of the single-CTA form.  Stage hand-over: the odd CTA's
-// transform and epilogue warps arrive directly on the even CTA's barriers, its MMA warp forwards
-// "my weights have landed", and stage releases come back by multicast commit.
+// epilogue warps arrive directly on the even CTA's barriers, its MMA warp forwards "my weights have
+// landed", its relay warp (warp 3) "my operand stage is written", and stage releases come back by
+// multicast commit.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -43,14 +44,15 @@ namespace {
 
 using namespace tc;
 
-// Warps: raw producer, weight producer, MMA issuer, 8 transform warps, then kEpi (8 or 4) epilogue warps.
-// With 8 epilogue warps the block has 608 threads and 96 registers per thread; with 4 it has 480 and
-// 128, which the transform warps (ten independent address chains, twenty values in flight) turn into
+// Warps: raw producer, weight producer, MMA issuer, relay, 8 transform warps, then kEpi (8 or 4) epilogue
+// warps.  With 8 epilogue warps the block has 640 threads and 96 registers per thread; with 4 it has 512
+// and 128, which the transform warps (ten independent address chains, twenty values in flight) turn into
 // speed: layers bound by the transform and with several tiles per CTA (so that the slower epilogue
 // hides behind the next tile) take the 4-warp form.
 constexpr int kXformWarps = 8;
 constexpr int kXformThreads = kXformWarps * 32;
-constexpr int kFirstXformWarp = 3, kFirstEpiWarp = kFirstXformWarp + kXformWarps;
+constexpr int kRelayWarp = 3;               // odd CTA of a pair: passes "operand stage written" on to the issuing CTA
+constexpr int kFirstXformWarp = 4, kFirstEpiWarp = kFirstXformWarp + kXformWarps;
 constexpr int threads_for(int epi_warps) { return (kFirstEpiWarp + epi_warps) * 32; }
 constexpr int kOwned = 10;                 // (slot, chunk) units of an A stage one transform thread may own
 constexpr int kMaxRawStages = 4;
@@ -64,6 +66,7 @@ static_assert(sizeof(TcConvSegs) <= kSegBytes, "segment table does not fit its s
 
 struct Bars {
     uint64_t raw_full[kMaxRawStages], raw_empty[kMaxRawStages], a_full[kMaxAStages], a_empty[kMaxAStages];
+    uint64_t a_done[kMaxAStages];            // odd CTA of a pair: its transform warps have written the stage
     uint64_t b_full[kMaxBStages], b_empty[kMaxBStages];
     uint64_t acc_full[2], acc_empty[2];
     uint64_t seg_full[2], seg_empty[2];      // segment tables, one per tile parity
@@ -147,7 +150,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             mbar_init(&bars->raw_empty[s], kXformWarps);
         }
         for (int s = 0; s < g.na_stages; ++s) {
-            mbar_init(&bars->a_full[s], kXformWarps * kCtas);      // waited on by the issuing CTA only
+            // waited on by the issuing CTA only: its own transform warps, plus one message from the peer
+            mbar_init(&bars->a_full[s], kCtas == 2 ? (g.relay ? kXformWarps + 1 : 2 * kXformWarps) : kXformWarps);
+            mbar_init(&bars->a_done[s], kXformWarps);
             mbar_init(&bars->a_empty[s], 1);
         }
         for (int s = 0; s < g.nb_stages; ++s) {
@@ -358,6 +363,27 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             }
             PROF_FLUSH(0);
         }
+    } else if (warp == kRelayWarp) {
+        // ------------------------------------------------------------ operand-stage relay (odd CTA of a pair)
+        // The issuing CTA's tensor core reads this CTA's operand stage, so the transform warps' writes must
+        // be released at cluster scope before the issuing CTA hears of them.  That fence stalls its thread
+        // for about a thousand cycles; done by each transform warp it cost them a quarter of their time.
+        // They arrive on a barrier of their own CTA instead (CTA scope: cheap), and this thread, which has
+        // nothing else to do, acquires that, fences at cluster scope (release is cumulative: it covers what
+        // it acquired) and arrives on the issuing CTA's barrier.
+        if (kCtas == 2 && rank != 0 && g.relay && elect_one()) {
+            const uint32_t peer_a_full = map_to_cta(smem_u32(&bars->a_full[0]), 0);
+            const int ncb = g.ncb, na = g.na_stages;
+            int as = 0;
+            uint32_t aphase = 0;
+            for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
+                for (int cb = 0; cb < ncb; ++cb) {
+                    mbar_wait(&bars->a_done[as], aphase, err, 22);
+                    mbar_arrive_remote_release(peer_a_full + (uint32_t)as * 8u);
+                    if (++as == na) { as = 0; aphase ^= 1; }
+                }
+            }
+        }
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------ transform warps
         const int xw = warp - kFirstXformWarp;     // 0..7
@@ -522,8 +548,12 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (kCtas == 2) mbar_arrive_remote_release(a_full_addr + (uint32_t)as * 8u);   // the issuing CTA's barrier
-                    else mbar_arrive(&bars->a_full[as]);
+                    if (kCtas == 2 && rank != 0) {
+                        if (g.relay) mbar_arrive(&bars->a_done[as]);                // the relay warp passes it on
+                        else mbar_arrive_remote_release(a_full_addr + (uint32_t)as * 8u);
+                    } else {
+                        mbar_arrive(&bars->a_full[as]);                             // the issuing CTA's own barrier
+                    }
                     mbar_arrive(&bars->raw_empty[rs]);
                 }
                 PROF_MARK(3);
@@ -807,6 +837,7 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
     // still leaves 64 KB for the weight ring.
     g.na_stages = 2;
     g.nr_stages = 2;
+    g.relay = 0;
     {
         // "ONNXB_CONV_STAGES=a,r" pins the operand / raw stage counts for A/B measurements
         int fa = 0, fr = 0;
@@ -814,6 +845,16 @@ bool fill_plan(const ConvGeom &c, int ctas, int MT, int BN, int KB, TcConvPlan &
         if (e && sscanf(e, "%d,%d", &fa, &fr) == 2 && fa >= 2 && fa <= kMaxAStages && fr >= 2 && fr < kMaxRawStages) {
             g.na_stages = fa;
             g.nr_stages = fr;
+        } else if (MT == 2 && g.KB >= 16 &&
+                   kSmemLimit - (1024 + 3LL * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes) -
+                           2LL * g.raw_stage_bytes >= 65536) {
+            // Two accumulators per CTA: a third operand stage instead of a third raw stage (64 -> 64
+            // channels at 56x56: 55.5 -> 52.3 us), and in a CTA pair the odd CTA's "stage written" message
+            // through its relay warp.  The message then arrives later, which three stages absorb, and the
+            // transform warps no longer wait for their cluster-scope fence (128 -> 128 channels at 28x28:
+            // 43.4 -> 41.0 us; with two stages the relay loses).
+            g.na_stages = 3;
+            g.relay = ctas == 2 ? 1 : 0;
         } else {
             const long long bf = 1024 + 2LL * g.a_stage_bytes + kMaxRawStages * kSegBytes + kBarBytes;
             for (int nr = 3; nr <= kMaxRawStages - 1; ++nr)
@@ -901,11 +942,16 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
         const double ring = (double)p.nb_stages * p.b_stage_bytes;
         const double t_w = std::max(w_bytes / std::min(48.0, 3600.0 / active), w_bytes * 2500.0 / ring);
         const double t_x = 300.0 + 100.0 * ((p.planes * p.SLOTS * p.nchunks + 255) / 256);
-        const double per_cb = std::max(std::max(t_mma, t_smem), std::max(t_w, t_x)) + 400.0 + (p.ctas == 2 ? 700.0 : 0.0);
+        // (three operand stages hide most of the hand-over)
+        const double per_cb = std::max(std::max(t_mma, t_smem), std::max(t_w, t_x)) +
+                              (p.na_stages == 3 ? 300.0 : 400.0 + (p.ctas == 2 ? 700.0 : 0.0));
         const bool dbl = p.MT == 1 || p.BN <= 128;
         const double t_epi = 8.0 * p.MT * p.BN;                             // read-back and stores of one tile
         const double per_tile = (dbl ? std::max(p.ncb * per_cb, t_epi) : p.ncb * per_cb + t_epi) + 3000.0;
-        const double cost = (double)waves * per_tile + 9000.0 + (dbl ? t_epi : 0.0);
+        double cost = (double)waves * per_tile + 9000.0 + (dbl ? t_epi : 0.0);
+        // pairs of 64-channel tiles with two accumulators measure 12-15 % slower than this model says
+        // (64 -> 64 channels at 56x56: 59 us against 52 us with one CTA per tile)
+        if (p.ctas == 2 && p.MT == 2 && p.BN <= 64 && p.KB >= 16) cost *= 1.15;
         if (!have || cost < best_cost * 0.999) {
             have = true;
             best_cost = cost;
@@ -921,6 +967,11 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
         plan.epi_warps = (plan.KB == 4 && plan.total_tiles >= 3LL * units) ? 4 : 8;
         if (const char *e = getenv("ONNXB_CONV_EPI"))
             if (e[0] == '4' || e[0] == '8') plan.epi_warps = e[0] - '0';
+        // Thin first layers in tap-pair mode are paced by the transform warps: take their fence off them too
+        // (ResNet-50 stem: 109.3 -> 106.6 us).  ONNXB_CONV_RELAY = 0 | 1 pins the choice for A/B measurements.
+        if (plan.ctas == 2 && plan.KB == 4) plan.relay = 1;
+        if (const char *e = getenv("ONNXB_CONV_RELAY"))
+            if (e[0] == '0' || e[0] == '1') plan.relay = e[0] - '0';
     }
     return have;
 }

@@ -69,6 +69,7 @@ struct TcConvPlan {
     ConvDivisor dv_L, dv_Ws, dv_Hs, dv_BOXP, dv_SLOTS, dv_pss;
     int boxp_shift;                  // log2(BOXP) when BOXP is a power of two, else -1
     int epi_warps;                   // epilogue warps of the launch: 8, or 4 (then 128 registers per thread)
+    int relay;                       // pairs: the odd CTA's "operand stage written" goes through its relay warp
 };
 
 // floor(n / d) for any 32-bit unsigned n.  On the device: the round-up multiply-and-shift method

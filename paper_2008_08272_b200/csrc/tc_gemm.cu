@@ -625,6 +625,10 @@ int launch_tc_gemm(const TcGemmProblem &g, void *stream) {
     const int units = p.ctas == 2 ? gemm_max_pairs() : sms;
     p.tiles_m = (g.M + kBM * p.ctas - 1) / (kBM * p.ctas);
     p.BN = pick_bn(p.tiles_m, g.N, g.batch, units, p.ctas);
+    if (const char *e = getenv("ONNXB_GEMM_BN")) {          // pins the tile width for A/B measurements
+        const int v = atoi(e);
+        if (v >= 32 * p.ctas && v <= kMaxBN && v % (32 * p.ctas) == 0) p.BN = v;
+    }
     p.BNH = p.BN / p.ctas;
     p.tiles_n = (g.N + p.BN - 1) / p.BN;
     p.num_kb = (g.K + kBK - 1) / kBK;

@@ -203,6 +203,31 @@ def test_conv_implicit_gemm_four_epilogue_warps(binding, c, monkeypatch):
     assert worst_ratio(got, want, S) <= 1.0
 
 
+@pytest.mark.parametrize("relay", ["0", "1"])
+@pytest.mark.parametrize("stages", ["2,2", "3,2"])
+@pytest.mark.parametrize("tile", ["2,1,64", "2,2,64"])
+def test_conv_implicit_gemm_pair_stage_handover(binding, tile, stages, relay, monkeypatch):
+    """CTA pairs: the odd CTA's "operand stage written" message straight from its transform warps or through
+    its relay warp, with two and three operand stages, on a problem with several tiles per CTA pair (so
+    that every barrier of the hand-over wraps its phase more than once)."""
+    rng = np.random.default_rng(int(relay) * 7 + len(tile))
+    xs, ws = (40, 32, 30, 30), (64, 32, 3, 3)            # 40 x 31 x 31 slots = 150 / 75 pair tiles of 256 / 512
+    X = rng.standard_normal(xs).astype(np.float32)
+    W = rng.standard_normal(ws).astype(np.float32)
+    B = rng.standard_normal((ws[0],)).astype(np.float32)
+    monkeypatch.setenv("ONNXB_CONV_TILE", tile)           # all three are read when the descriptor is created
+    monkeypatch.setenv("ONNXB_CONV_STAGES", stages)
+    monkeypatch.setenv("ONNXB_CONV_RELAY", relay)
+    binding.set_kernel_override("mma_implicit")
+    try:
+        got, fam = run_conv_gpu(binding, torch, X, W, B, relu=True, pads=(1, 1, 1, 1))
+    finally:
+        binding.set_kernel_override(None)
+    assert fam == "mma_implicit"
+    want, S = oracle.conv2d(X, W, B, relu=True, pads=(1, 1, 1, 1))
+    assert worst_ratio(got, want, S) <= 1.0
+
+
 @pytest.mark.parametrize("pair", ["0", "1"])
 @pytest.mark.parametrize("shape", [(256, 200, 96), (384, 3136, 64), (300, 260, 130), (512, 64, 1024)])
 def test_gemm_cta_pair_choice(binding, shape, pair, monkeypatch):
