@@ -952,6 +952,9 @@ bool tc_conv_plan(const ConvGeom &c, TcConvPlan &plan, bool forced) {
         // pairs of 64-channel tiles with two accumulators measure 12-15 % slower than this model says
         // (64 -> 64 channels at 56x56: 59 us against 52 us with one CTA per tile)
         if (p.ctas == 2 && p.MT == 2 && p.BN <= 64 && p.KB >= 16) cost *= 1.15;
+        // tap-pair mode (thin first layers) streams hardly any weights, so a pair shares nothing worth its
+        // hand-over (ResNet-50 stem: 106.8 us as pairs, 101.8 us with one CTA per tile)
+        if (p.ctas == 2 && p.KB == 4) cost *= 1.15;
         if (!have || cost < best_cost * 0.999) {
             have = true;
             best_cost = cost;
