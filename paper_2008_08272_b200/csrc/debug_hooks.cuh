@@ -11,8 +11,8 @@ __device__ long long g_prof[148 * 16];
 #define PROF_DECL long long pt_ = clock64(), pacc_[6] = {0, 0, 0, 0, 0, 0}
 #define PROF_MARK(k) do { long long n_ = clock64(); pacc_[k] += n_ - pt_; pt_ = n_; } while (0)
 #define PROF_FLUSH(base) do { if (blockIdx.x < 148) for (int k_ = 0; k_ < 6; ++k_) g_prof[blockIdx.x * 16 + (base) + k_] = pacc_[k_]; } while (0)
-// event log of CTA 0: kind k (0..7), sequence number i (0..63) -> clock
-__device__ long long g_log[8 * 64];
+// event log of CTA 0: kind k (0..8; 8 = phases of the kernel as a whole), sequence number i (0..63) -> clock
+__device__ long long g_log[9 * 64];
 #define LOG(k, i) do { if (blockIdx.x == 0 && (i) < 64) g_log[(k) * 64 + (i)] = clock64(); } while (0)
 extern "C" int onnxb_dbg_profile(long long *out) {
     cudaDeviceSynchronize();
@@ -23,7 +23,7 @@ extern "C" int onnxb_dbg_profile(long long *out) {
 }
 extern "C" int onnxb_dbg_log(long long *out) {
     cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out, g_log, sizeof(long long) * 8 * 64);
+    cudaMemcpyFromSymbol(out, g_log, sizeof(long long) * 9 * 64);
     return 0;
 }
 #else

@@ -135,6 +135,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     Bars *bars = reinterpret_cast<Bars *>(seg_st + kMaxRawStages * kSegBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) LOG(8, 0);
     const int tile_rows = g.MT * 128;
     // CTA pair: rank within the cluster, and the tiles this CTA (pair) walks
     const uint32_t rank = kCtas == 2 ? cluster_ctarank() : 0u;
@@ -179,7 +180,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     const uint32_t tmem_base = bars->tmem_holder;
     if (kCtas == 2) cluster_sync_all();     // the peer's barriers exist before anything arrives on them
     pdl_launch_dependents();
-    pdl_wait();                 // everything above overlapped the previous kernel's tail
+    // Everything above overlapped the previous kernel's tail, and so does each role's own set-up below:
+    // the threads that touch global memory (the two producers, the epilogue warps) wait for the previous
+    // kernel just before their first access; the others only ever see what those threads hand them.
 
     if (warp == 0) {
         // ------------------------------------------------------------ raw activation producer
@@ -202,6 +205,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
                 tc_conv_segments(g, G0, *segs);
                 mbar_arrive(&bars->seg_full[sp]);
                 ++tile_it;
+                if (tile_it == 1) {
+                    pdl_wait();
+                    LOG(8, 1);
+                }
                 const int nseg = segs->nseg;
                 const uint32_t tile_bytes = (uint32_t)segs->total_floats * 4u;
                 const int rot = cb_rotation(t, ncb);
@@ -252,6 +259,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             const long long per_ct = (long long)g.ncb * g.n_steps * g.b_step_bytes;   // bytes per channel tile and CTA
             const int nb = g.nb_stages, ncb = g.ncb, b_steps = g.b_steps, spb = g.spb, n_steps = g.n_steps;
             const uint32_t stage_bytes = (uint32_t)g.b_stage_bytes, step_bytes = (uint32_t)g.b_step_bytes;
+            pdl_wait();             // the packed weights may come from the kernel just before this one
             for (long long t = first_tile; t < g.total_tiles; t += tile_step) {
                 const int ct_all = (int)(t % cgt);
                 const uint8_t *tile_src = reinterpret_cast<const uint8_t *>(Wpk) + (ct_all * kCtas + (int)rank) * per_ct;
@@ -579,6 +587,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             const uint32_t ab = acc_dbl ? (it & 1u) : 0u, use = acc_dbl ? (it >> 1) : it;
             mbar_wait(&bars->acc_full[ab], use & 1u, err, 18);
             tc_fence_after_sync();
+            if (it == 0) pdl_wait();        // long since satisfied: the producers passed theirs before the first load
+            if (ew == 0 && lane == 0) LOG(8, 2);
             const int nch = (g.BN + 31) / 32;
             // eight warps: two per TMEM lane quarter, each taking half of the tile; four: one per quarter, both halves
             for (int hf = ew >> 2; hf < 2; hf += kEpiWarps / 4) {
@@ -618,6 +628,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
             }
             tc_fence_before_sync();
             __syncwarp();
+            if (ew == 0 && lane == 0) LOG(8, 3);
             if (lane == 0) {
                 if (kCtas == 2) mbar_arrive_remote(acc_empty_addr + ab * 8u);
                 else mbar_arrive(&bars->acc_empty[ab]);
@@ -628,6 +639,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap tmX, const TcConvPlan g, cons
     tc_fence_before_sync();
     __syncthreads();
     if (kCtas == 2) cluster_sync_all();     // no CTA leaves while its peer may still signal it
+    if (threadIdx.x == 0) LOG(8, 4);
     if (warp == 2) {
         __syncwarp();
         tc_fence_after_sync();

@@ -134,7 +134,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tmem_base = *tmem_holder;
     if (kCtas == 2) cluster_sync_all();     // the peer's barriers exist before anything arrives on them
     pdl_launch_dependents();
-    pdl_wait();                 // everything above overlapped the previous kernel's tail
+    // Everything above overlapped the previous kernel's tail, and so does each role's own set-up below: the
+    // warps that touch global memory (the producer, the epilogue warps) wait for the previous kernel just
+    // before their first access; the MMA warp only ever sees what the producer hands it.
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -197,6 +199,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     c2 = bb;
                     d1 = kBK;
                 }
+                if (t == first_tile) pdl_wait();
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     mbar_wait(&empty[stage], phase ^ 1, p.err, 1);
                     if (lane == 0) GLOG(0, glog_i++);
@@ -287,6 +290,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------------------ epilogue
+        pdl_wait();
         const int q = warp & 3;                    // TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;          // which half of the tile's 32-column blocks
         uint8_t *buf = staging + (warp - 2) * kStoreBufBytes;
