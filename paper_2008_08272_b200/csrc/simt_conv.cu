@@ -270,6 +270,7 @@ conv2d_depthwise_unit_kernel(const ConvGeom g, const float *__restrict__ X, cons
                              const float *__restrict__ B, const float *__restrict__ R, float *__restrict__ Y,
                              unsigned items, unsigned Q4, unsigned P2, double inv_Q4, double inv_P2) {
     constexpr int WIN = KW + 3;                // input columns a strip of 4 outputs touches
+    tc::pdl_launch_dependents();               // (launched plainly itself) lets the next kernel set up early
     const unsigned i = blockIdx.x * 256u + threadIdx.x;
     if (i >= items) return;
     // i = (plane * P2 + row group) * Q4 + column quad (P2 = row groups per plane); quotients by reciprocal multiplication in
